@@ -1,0 +1,278 @@
+/*
+ * cwlo.c -- fp64 CPU oracle for the ChunkWise-LoRA hot path (TEST INFRASTRUCTURE ONLY).
+ * See cwlo.h for scope, citations and pin status.  No blocking, no fusion, no BLAS: every
+ * function is the definition (or the algorithm's steps in order) written out.
+ */
+#include "cwlo.h"
+
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define Q24 16777216 /* 2^24 */
+
+int cwlo_get_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+void cwlo_set_threads(int n) {
+#ifdef _OPENMP
+  if (n >= 1) omp_set_num_threads(n);
+#else
+  (void)n;
+#endif
+}
+
+/* ---------------------------------------------------------------------------------------------
+ * Sec. III-A signal (i): next-token entropy of softmax(z), normalised by ln V so that the
+ * thresholds of the selector live in [0,1].
+ *   m = max z;  S = sum exp(z-m);  U = sum (z-m) exp(z-m);  H = ln S - U/S;  score = H / ln V.
+ * A -inf logit has probability zero and contributes nothing.  A row holding NaN or +inf, or
+ * made of -inf only, has no defined entropy: NaN (the chunker treats NaN as hardest).
+ * ------------------------------------------------------------------------------------------- */
+static double entropy_row(const float* z, int32_t V) {
+  double m = -INFINITY;
+  for (int32_t v = 0; v < V; ++v) {
+    double zv = (double)z[v];
+    if (isnan(zv) || zv == INFINITY) return NAN;
+    if (zv > m) m = zv;
+  }
+  if (m == -INFINITY) return NAN;
+  double S = 0.0, U = 0.0;
+  for (int32_t v = 0; v < V; ++v) {
+    double zv = (double)z[v];
+    if (zv == -INFINITY) continue;
+    double d = zv - m;
+    double e = exp(d);
+    S += e;
+    U += d * e;
+  }
+  double H = log(S) - U / S;
+  double s = H / log((double)V);
+  if (s < 0.0) s = 0.0;
+  if (s > 1.0) s = 1.0;
+  return s;
+}
+
+int cwlo_score_tokens(const float* logits, int64_t ld, int32_t T, int32_t V, double* score) {
+  if (!logits || !score || T < 0 || V < 2 || ld < V) return CWLO_ERR_ARG;
+#pragma omp parallel for schedule(static)
+  for (int32_t t = 0; t < T; ++t) score[t] = entropy_row(logits + (int64_t)t * ld, V);
+  return CWLO_OK;
+}
+
+/* ---------------------------------------------------------------------------------------------
+ * Sec. III-B "average-complexity threshold": chunk means are compared in fixed point so that
+ * the partition is a function of the fp32 score array alone, independent of summation order.
+ * ------------------------------------------------------------------------------------------- */
+int64_t cwlo_quantise(float s) {
+  if (isnan(s)) return Q24;
+  double c = (double)s;
+  if (c < 0.0) c = 0.0;
+  if (c > 1.0) c = 1.0;
+  return (int64_t)floor(c * (double)Q24);
+}
+
+static int64_t threshold_q(float theta) { return (int64_t)floor((double)theta * (double)Q24); }
+
+/* Sec. III-C / IV-C rule-based mapping: the rung is the number of thresholds the chunk mean
+ * reaches (mean >= theta_k  <=>  sum >= Theta_k * len). */
+int32_t cwlo_rung(int64_t sum, int64_t len, const cwlo_policy* p) {
+  int32_t k = 0;
+  for (int32_t j = 0; j + 1 < p->n_rungs; ++j)
+    if (sum >= threshold_q(p->threshold[j]) * len) ++k;
+  return k;
+}
+
+static int policy_ok(const cwlo_policy* p) {
+  if (!p || p->n_rungs < 1 || p->n_rungs > CWLO_MAX_RUNGS) return 0;
+  if (p->min_len < 1 || p->max_len < p->min_len) return 0;
+  if ((int64_t)p->min_len + (int64_t)p->max_len > (1 << 19)) return 0;
+  if (p->window < 0 || p->window > p->min_len) return 0;
+  for (int32_t k = 0; k < p->n_rungs; ++k) {
+    if (p->rung_rank[k] < 0) return 0;
+    if (k > 0 && p->rung_rank[k] < p->rung_rank[k - 1]) return 0;
+  }
+  for (int32_t k = 0; k + 1 < p->n_rungs; ++k) {
+    float th = p->threshold[k];
+    if (!(th >= 0.0f && th <= 1.0f)) return 0;
+    if (k > 0 && !(th > p->threshold[k - 1])) return 0;
+  }
+  return 1;
+}
+
+int cwlo_partition(const float* score, const int32_t* cu, int32_t n_seq, int32_t T,
+                   const cwlo_policy* p, int32_t* offsets, int32_t* rank, float* scale,
+                   int32_t* rung, int32_t* flags, int32_t* n_chunks, int32_t capacity) {
+  if (!score || !cu || !offsets || !rank || !scale || !rung || !flags || !n_chunks) return CWLO_ERR_ARG;
+  if (n_seq < 0 || T < 0 || capacity < 0 || !policy_ok(p)) return CWLO_ERR_ARG;
+  if (cu[0] != 0 || cu[n_seq] != T) return CWLO_ERR_ARG;
+  for (int32_t n = 0; n < n_seq; ++n)
+    if (cu[n + 1] < cu[n]) return CWLO_ERR_ARG;
+
+  /* exclusive prefix sums of the quantised scores */
+  int64_t* P = (int64_t*)malloc(sizeof(int64_t) * ((size_t)T + 1));
+  if (!P) return CWLO_ERR_ARG;
+  P[0] = 0;
+  for (int32_t t = 0; t < T; ++t) P[t + 1] = P[t] + cwlo_quantise(score[t]);
+
+  const int32_t Lmin = p->min_len, Lmax = p->max_len, K = p->n_rungs;
+  int32_t C = 0;
+  int status = CWLO_OK;
+  offsets[0] = 0;
+
+  for (int32_t n = 0; n < n_seq && status == CWLO_OK; ++n) {
+    const int32_t S = cu[n], E = cu[n + 1];
+    const int32_t first_chunk = C;
+    /* -- the greedy online walk (Sec. III-B): grow the open chunk one token at a time, close it
+     *    at the length cap or where the next L_min tokens fall in another complexity class -- */
+    int32_t b = S;
+    while (b < E) {
+      int32_t e;
+      if (E - b < 2 * Lmin) {
+        e = E; /* two legal chunks do not fit: take the rest */
+      } else {
+        e = b + Lmin;
+        for (;;) {
+          if (e - b >= Lmax) break;
+          int32_t open_rung  = cwlo_rung(P[e] - P[b], e - b, p);
+          int32_t ahead_rung = cwlo_rung(P[e + Lmin] - P[e], Lmin, p);
+          if (open_rung != ahead_rung) break;
+          e = e + 1;
+          if (E - e < Lmin) { e = E; break; } /* the tail would be too short: absorb it */
+        }
+      }
+      if (C >= capacity) { status = CWLO_ERR_CAPACITY; break; }
+      offsets[C + 1] = e;
+      flags[C] = (b == S) ? 1 : 0;
+      rung[C] = cwlo_rung(P[e] - P[b], e - b, p);
+      ++C;
+      b = e;
+    }
+    if (status != CWLO_OK) break;
+
+    /* -- budget on high-capacity regions (Sec. III-B): at most hi_budget chunks of this
+     *    sequence stay on the top rung; the ones with the smallest means step down one rung -- */
+    if (p->hi_budget >= 0 && K >= 2 && C > first_chunk) {
+      /* the ranking is taken over the rungs as the walk left them, before any demotion */
+      int32_t* walked = (int32_t*)malloc(sizeof(int32_t) * (size_t)(C - first_chunk));
+      for (int32_t c = first_chunk; c < C; ++c) walked[c - first_chunk] = rung[c];
+      for (int32_t c = first_chunk; c < C; ++c) {
+        if (walked[c - first_chunk] != K - 1) continue;
+        int64_t sum_c = P[offsets[c + 1]] - P[offsets[c]], len_c = offsets[c + 1] - offsets[c];
+        int32_t better = 0; /* top-rung chunks of this sequence that outrank chunk c */
+        for (int32_t d = first_chunk; d < C; ++d) {
+          if (d == c || walked[d - first_chunk] != K - 1) continue;
+          int64_t sum_d = P[offsets[d + 1]] - P[offsets[d]], len_d = offsets[d + 1] - offsets[d];
+          int64_t lhs = sum_d * len_c, rhs = sum_c * len_d; /* mean_d against mean_c */
+          if (lhs > rhs || (lhs == rhs && d < c)) ++better;
+        }
+        if (better >= p->hi_budget) rung[c] = K - 2;
+      }
+      free(walked);
+    }
+  }
+
+  if (status == CWLO_OK) {
+    for (int32_t c = 0; c < C; ++c) {
+      rank[c] = p->rung_rank[rung[c]];
+      scale[c] = p->rung_scale[rung[c]];
+    }
+    *n_chunks = C;
+  }
+  free(P);
+  return status;
+}
+
+/* ---------------------------------------------------------------------------------------------
+ * Sec. III-D: over a short window after a join the outgoing adapter ramps down linearly while
+ * the incoming one ramps up.  The window is the first w rows of the incoming chunk; the ramp
+ * takes the w equally spaced values strictly between 0 and 1.
+ * ------------------------------------------------------------------------------------------- */
+double cwlo_blend_weight(int32_t t, const int32_t* offsets, const int32_t* flags,
+                         int32_t n_chunks, int32_t window, int32_t* chunk) {
+  int32_t c = 0;
+  while (c + 1 < n_chunks && offsets[c + 1] <= t) ++c;
+  if (chunk) *chunk = c;
+  int32_t j = t - offsets[c];
+  if (c == 0 || (flags[c] & 1) || j >= window) return 1.0;
+  return (double)(j + 1) / (double)(window + 1);
+}
+
+static double bf16_to_double(uint16_t h) {
+  uint32_t u = ((uint32_t)h) << 16;
+  float f;
+  memcpy(&f, &u, sizeof f);
+  return (double)f;
+}
+
+/* delta[n] = s * sum_{j<r} (sum_k x[k] A[k,j]) B[j,n]   -- one adapter configuration, one row */
+static void adapter_row(const uint16_t* x, const uint16_t* A, int64_t lda, const uint16_t* B,
+                        int64_t ldb, int32_t d_in, int32_t d_out, int32_t r, double s,
+                        double* h, double* delta) {
+  for (int32_t n = 0; n < d_out; ++n) delta[n] = 0.0;
+  for (int32_t j = 0; j < r; ++j) {
+    double acc = 0.0;
+    for (int32_t k = 0; k < d_in; ++k) acc += bf16_to_double(x[k]) * bf16_to_double(A[(int64_t)k * lda + j]);
+    h[j] = acc;
+  }
+  for (int32_t j = 0; j < r; ++j)
+    for (int32_t n = 0; n < d_out; ++n) delta[n] += h[j] * bf16_to_double(B[(int64_t)j * ldb + n]);
+  for (int32_t n = 0; n < d_out; ++n) delta[n] *= s;
+}
+
+int cwlo_apply(const uint16_t* X, int64_t ldx, const uint16_t* W, int64_t ldw,
+               const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
+               int32_t T, int32_t d_in, int32_t d_out, int32_t R,
+               const int32_t* offsets, const int32_t* rank, const float* scale,
+               const int32_t* flags, int32_t n_chunks, int32_t window,
+               const int32_t* rows, int32_t n_rows, double* Y, int64_t ldy) {
+  if (!X || !W || !Y || T < 0 || d_in < 1 || d_out < 1 || R < 0 || window < 0) return CWLO_ERR_ARG;
+  const int has_adapter = (A != NULL && B != NULL && R > 0);
+  if (has_adapter) {
+    if (!offsets || !rank || !scale || !flags || n_chunks < 1) return CWLO_ERR_ARG;
+    if (offsets[0] != 0 || offsets[n_chunks] != T) return CWLO_ERR_ARG;
+    for (int32_t c = 0; c < n_chunks; ++c)
+      if (rank[c] < 0 || rank[c] > R || offsets[c + 1] < offsets[c]) return CWLO_ERR_ARG;
+  }
+  const int32_t count = rows ? n_rows : T;
+  int bad = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int32_t i = 0; i < count; ++i) {
+    const int32_t t = rows ? rows[i] : i;
+    if (t < 0 || t >= T) { bad = 1; continue; }
+    const uint16_t* x = X + (int64_t)t * ldx;
+    double* y = Y + (int64_t)i * ldy;
+    /* base projection x_t W */
+    for (int32_t n = 0; n < d_out; ++n) y[n] = 0.0;
+    for (int32_t k = 0; k < d_in; ++k) {
+      double xk = bf16_to_double(x[k]);
+      const uint16_t* w = W + (int64_t)k * ldw;
+      for (int32_t n = 0; n < d_out; ++n) y[n] += xk * bf16_to_double(w[n]);
+    }
+    if (!has_adapter) continue;
+    int32_t c;
+    double lam = cwlo_blend_weight(t, offsets, flags, n_chunks, window, &c);
+    double* h = (double*)malloc(sizeof(double) * (size_t)(R > 0 ? R : 1));
+    double* d_in_c = (double*)malloc(sizeof(double) * (size_t)d_out);
+    double* d_out_p = (double*)malloc(sizeof(double) * (size_t)d_out);
+    /* incoming (own chunk) adapter output */
+    adapter_row(x, A, lda, B, ldb, d_in, d_out, rank[c], (double)scale[c], h, d_in_c);
+    if (lam < 1.0) {
+      /* outgoing (previous chunk) adapter output, then the literal cross-fade */
+      adapter_row(x, A, lda, B, ldb, d_in, d_out, rank[c - 1], (double)scale[c - 1], h, d_out_p);
+      for (int32_t n = 0; n < d_out; ++n) y[n] += (1.0 - lam) * d_out_p[n] + lam * d_in_c[n];
+    } else {
+      for (int32_t n = 0; n < d_out; ++n) y[n] += d_in_c[n];
+    }
+    free(h); free(d_in_c); free(d_out_p);
+  }
+  return bad ? CWLO_ERR_ARG : CWLO_OK;
+}
