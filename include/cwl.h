@@ -1,0 +1,131 @@
+/*
+ * cwl.h -- C ABI of the B200 (sm_100a) ChunkWise-LoRA hot path.
+ *
+ * Three calls follow the paper's pipeline (Sec. III):
+ *   cwl_score_tokens  token complexity estimator, entropy signal        (Sec. III-A (i), IV-A)
+ *   cwl_partition     adaptive chunker + per-chunk rank/scale selector  (Sec. III-B, III-C, IV-B, IV-C)
+ *   cwl_apply         adapted projection with the boundary cross-fade   (Sec. III-D, III-F, IV-E)
+ *
+ * Conventions for every call
+ *   - Pointers marked DEV are device pointers owned by the caller; the library never frees or
+ *     keeps them.  Pointers marked HOST are read during the call only.
+ *   - All matrices are row-major with an explicit leading dimension in ELEMENTS.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Work is
+ *     enqueued on it and the call returns without synchronising.
+ *   - Argument errors are reported synchronously through the return value and nothing is
+ *     launched.  Problems only visible on the device (chunk table capacity exceeded, a bounded
+ *     wait that ran out) are OR-ed as (1 << status) into *status_word (DEV int32, may be NULL);
+ *     the caller zeroes it.  The library never traps, prints or exits.
+ *   - Calls on distinct streams may run concurrently as long as they use distinct workspaces.
+ *   - The library allocates no device memory in these calls; scratch comes from `workspace`.
+ */
+#ifndef CWL_H
+#define CWL_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  CWL_OK = 0,
+  CWL_ERR_INVALID_ARG = 1, /* NULL pointer, negative size, malformed policy */
+  CWL_ERR_SHAPE = 2,       /* leading dimension smaller than the row, misaligned pointer or stride */
+  CWL_ERR_UNSUPPORTED = 3, /* shape outside the supported set (see each call) */
+  CWL_ERR_CAPACITY = 4,    /* chunk table too small (device-side, via status_word) */
+  CWL_ERR_WORKSPACE = 5,   /* workspace NULL or smaller than *_workspace_bytes() */
+  CWL_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed */
+  CWL_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out (device-side, via status_word) */
+} cwl_status;
+
+#define CWL_MAX_RUNGS 8
+#define CWL_MAX_RANK 256
+
+/* Chunker and selector policy (HOST, copied at call time).  The paper names these knobs
+ * (length bounds, average-complexity threshold, budget of high-capacity regions: Sec. III-B;
+ * rank ladder and gating scale: Sec. III-C) without giving values. */
+typedef struct {
+  int32_t n_rungs;                      /* K, 1..CWL_MAX_RUNGS */
+  int32_t rung_rank[CWL_MAX_RUNGS];     /* prefix rank of each rung, non-decreasing, >= 0 */
+  float   rung_scale[CWL_MAX_RUNGS];    /* gating scale of each rung (e.g. alpha / rank) */
+  float   threshold[CWL_MAX_RUNGS - 1]; /* strictly increasing, in [0,1]: mean >= threshold[k] climbs to rung k+1 */
+  int32_t min_len, max_len;             /* 1 <= min_len <= max_len, min_len + max_len <= 2^19 */
+  int32_t window;                       /* cross-fade window, 0 <= window <= min_len */
+  int32_t hi_budget;                    /* max top-rung chunks per sequence; < 0 = unlimited */
+} cwl_policy;
+
+/* Chunk table: struct of DEV arrays with `capacity` entries (`offsets` has capacity + 1).
+ * Chunk c covers rows [offsets[c], offsets[c+1]); offsets[0] = 0, offsets[n_chunks] = T. */
+typedef struct {
+  int32_t* offsets;  /* DEV int32 [capacity + 1] */
+  int32_t* rank;     /* DEV int32 [capacity]  prefix rank r_c */
+  float*   scale;    /* DEV fp32  [capacity]  gating scale s_c */
+  int32_t* rung;     /* DEV int32 [capacity]  ladder index (written by cwl_partition, unused by cwl_apply) */
+  int32_t* flags;    /* DEV int32 [capacity]  bit0 = first chunk of its sequence (never blended in) */
+  int32_t* n_chunks; /* DEV int32 [1] */
+  int32_t  capacity;
+} cwl_chunk_table;
+
+const char* cwl_status_string(cwl_status s);
+int         cwl_version(void);
+
+/* Token complexity score (Sec. III-A signal (i)): normalised entropy of softmax(logits[t, :]),
+ *   score[t] = (ln S - U / S) / ln V,  S = sum exp(z - max z),  U = sum (z - max z) exp(z - max z),
+ * clamped to [0,1].  -inf logits contribute nothing; a row with NaN or +inf, or of -inf only,
+ * scores NaN.  fp32 arithmetic.
+ *   logits DEV fp32 [T, V], row stride ld_logits >= V;  score DEV fp32 [T].
+ * Errors: INVALID_ARG (NULL, T < 0, V < 2), SHAPE (ld_logits < V).  T == 0 is a no-op. */
+cwl_status cwl_score_tokens(const float* logits, int64_t ld_logits, int32_t T, int32_t V,
+                            float* score, void* stream);
+
+/* Adaptive chunker and rank-ladder selector (Sec. III-B, III-C).
+ * Scores are quantised to q = floor(clamp(s,0,1) * 2^24) (NaN -> 2^24) and every mean is compared
+ * as an integer sum, so the result depends on the fp32 score array only.  Per sequence a greedy
+ * online walk closes the open chunk [b, e) at the first e >= b + min_len, with at least min_len
+ * tokens left after it, where e - b >= max_len or the rung of [b, e) differs from the rung of the
+ * look-ahead window [e, e + min_len); if fewer than 2 * min_len tokens remain, or no such e
+ * exists, the chunk takes the rest of the sequence.  rung = number of thresholds the mean reaches.
+ * With hi_budget = H >= 0 only the H top-rung chunks of a sequence with the largest means (earlier
+ * chunk first on ties) stay on the top rung; the others step down one rung.
+ *   score       DEV fp32 [T]
+ *   cu_seqlens  DEV int32 [n_seq + 1], cu[0] = 0, cu[n_seq] = T, non-decreasing (unchecked on device:
+ *               the caller guarantees it; empty sequences emit no chunk)
+ *   table       outputs; *n_chunks <= T / min_len + n_seq entries are needed.  If capacity is
+ *               too small, n_chunks is set to 0 and CWL_ERR_CAPACITY is flagged in *status_word.
+ *   workspace   DEV, at least cwl_partition_workspace_bytes(T, n_seq) bytes, 16-byte aligned
+ * Errors: INVALID_ARG (NULLs, bad policy, T < 0, n_seq < 0), WORKSPACE. */
+size_t     cwl_partition_workspace_bytes(int32_t T, int32_t n_seq);
+cwl_status cwl_partition(const float* score, const int32_t* cu_seqlens, int32_t n_seq, int32_t T,
+                         const cwl_policy* policy, cwl_chunk_table table,
+                         void* workspace, size_t workspace_bytes,
+                         int32_t* status_word, void* stream);
+
+/* Adapted projection (Sec. III-F) with the boundary-safe cross-fade (Sec. III-D):
+ *   y_t = x_t W + (1 - lam_t) s_p (x_t A[:, :r_p]) B[:r_p, :] + lam_t s_c (x_t A[:, :r_c]) B[:r_c, :]
+ * for row t in chunk c with predecessor p = c - 1.  Rows j = 0..window-1 of a chunk that is not
+ * first of its sequence have lam = (j + 1) / (window + 1); every other row has lam = 1.
+ * bf16 operands, fp32 accumulation on the tensor cores, bf16 (round-to-nearest-even) output.
+ *   X DEV bf16 [T, d_in]; W DEV bf16 [d_in, d_out]; A DEV bf16 [d_in, R]; B DEV bf16 [R, d_out];
+ *   Y DEV bf16 [T, d_out].  A == NULL or B == NULL or R == 0 computes the plain projection X W
+ *   (table is then ignored).
+ *   table       input; rows outside every chunk get no adapter.  rank[c] must lie in [0, R].
+ *   workspace   DEV, at least cwl_apply_workspace_bytes(T, d_in, d_out, R) bytes, 256-byte aligned
+ * Supported shapes: d_in, d_out, R multiples of 16; R <= CWL_MAX_RANK; all base pointers 16-byte
+ * aligned and leading dimensions multiples of 8 elements.  Anything else is CWL_ERR_UNSUPPORTED /
+ * CWL_ERR_SHAPE -- there is no slow path.
+ * Errors: INVALID_ARG, SHAPE, UNSUPPORTED, WORKSPACE, CUDA.  T == 0 is a no-op. */
+size_t     cwl_apply_workspace_bytes(int32_t T, int32_t d_in, int32_t d_out, int32_t R);
+cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64_t ldw,
+                     const void* A, int64_t lda, const void* B, int64_t ldb,
+                     int32_t T, int32_t d_in, int32_t d_out, int32_t R,
+                     cwl_chunk_table table, int32_t window,
+                     void* Y, int64_t ldy,
+                     void* workspace, size_t workspace_bytes,
+                     int32_t* status_word, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CWL_H */

@@ -1,0 +1,213 @@
+"""ctypes binding of libcwl.so: argument marshalling only.
+
+Every step of the path (scoring, partition, shrink, gate, projection) runs in the CUDA library;
+torch is used for device memory and streams.  There is no CPU fallback: if the library has not
+been built, loading raises.  Function names mirror the C ABI declared in ``include/cwl.h``.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcwl.so")
+MAX_RUNGS = 8
+
+STATUS = {0: "CWL_OK", 1: "CWL_ERR_INVALID_ARG", 2: "CWL_ERR_SHAPE", 3: "CWL_ERR_UNSUPPORTED",
+          4: "CWL_ERR_CAPACITY", 5: "CWL_ERR_WORKSPACE", 6: "CWL_ERR_CUDA", 7: "CWL_ERR_TIMEOUT"}
+
+EXPORTS = ["cwl_status_string", "cwl_version", "cwl_score_tokens", "cwl_partition_workspace_bytes",
+           "cwl_partition", "cwl_apply_workspace_bytes", "cwl_apply"]
+
+
+class CwlError(RuntimeError):
+    def __init__(self, call: str, status: int):
+        self.status = status
+        super().__init__(f"{call} failed: {STATUS.get(status, status)}")
+
+
+class CPolicy(C.Structure):
+    _fields_ = [("n_rungs", C.c_int32),
+                ("rung_rank", C.c_int32 * MAX_RUNGS),
+                ("rung_scale", C.c_float * MAX_RUNGS),
+                ("threshold", C.c_float * (MAX_RUNGS - 1)),
+                ("min_len", C.c_int32), ("max_len", C.c_int32),
+                ("window", C.c_int32), ("hi_budget", C.c_int32)]
+
+
+class CChunkTable(C.Structure):
+    _fields_ = [("offsets", C.c_void_p), ("rank", C.c_void_p), ("scale", C.c_void_p),
+                ("rung", C.c_void_p), ("flags", C.c_void_p), ("n_chunks", C.c_void_p),
+                ("capacity", C.c_int32)]
+
+
+_lib = None
+
+
+def lib():
+    """Loads libcwl.so (built by ``paper_2601_21109_b200.build``); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2601_21109_b200.build` "
+                               "(there is no fallback path)")
+        L = C.CDLL(LIB_PATH)
+        L.cwl_status_string.restype = C.c_char_p
+        L.cwl_status_string.argtypes = [C.c_int]
+        L.cwl_version.restype = C.c_int
+        L.cwl_score_tokens.restype = C.c_int
+        L.cwl_score_tokens.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        L.cwl_partition_workspace_bytes.restype = C.c_size_t
+        L.cwl_partition_workspace_bytes.argtypes = [C.c_int32, C.c_int32]
+        L.cwl_partition.restype = C.c_int
+        L.cwl_partition.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(CPolicy), CChunkTable,
+                                    C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        L.cwl_apply_workspace_bytes.restype = C.c_size_t
+        L.cwl_apply_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32]
+        L.cwl_apply.restype = C.c_int
+        L.cwl_apply.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
+                                C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                CChunkTable, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t,
+                                C.c_void_p, C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def _p(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else int(t.data_ptr())
+
+
+def make_policy(ranks: Sequence[int], scales: Sequence[float], thresholds: Sequence[float],
+                min_len: int, max_len: int, window: int, hi_budget: int = -1) -> CPolicy:
+    p = CPolicy()
+    p.n_rungs = len(ranks)
+    for k, r in enumerate(ranks):
+        p.rung_rank[k] = int(r)
+    for k, s in enumerate(scales):
+        p.rung_scale[k] = float(s)
+    for k, th in enumerate(thresholds):
+        p.threshold[k] = float(th)
+    p.min_len, p.max_len, p.window, p.hi_budget = int(min_len), int(max_len), int(window), int(hi_budget)
+    return p
+
+
+class DeviceChunkTable:
+    """Chunk table as device arrays (struct of arrays, as the C ABI takes it)."""
+
+    def __init__(self, capacity: int, device="cuda"):
+        self.capacity = int(capacity)
+        self.offsets = torch.zeros(self.capacity + 1, dtype=torch.int32, device=device)
+        self.rank = torch.zeros(max(self.capacity, 1), dtype=torch.int32, device=device)
+        self.scale = torch.zeros(max(self.capacity, 1), dtype=torch.float32, device=device)
+        self.rung = torch.zeros(max(self.capacity, 1), dtype=torch.int32, device=device)
+        self.flags = torch.zeros(max(self.capacity, 1), dtype=torch.int32, device=device)
+        self.n_chunks = torch.zeros(1, dtype=torch.int32, device=device)
+
+    @staticmethod
+    def from_host(offsets, rank, scale, flags, rung=None, device="cuda") -> "DeviceChunkTable":
+        n = len(rank)
+        t = DeviceChunkTable(n, device)
+        t.offsets.copy_(torch.as_tensor(offsets, dtype=torch.int32))
+        if n:
+            t.rank[:n].copy_(torch.as_tensor(rank, dtype=torch.int32))
+            t.scale[:n].copy_(torch.as_tensor(scale, dtype=torch.float32))
+            t.flags[:n].copy_(torch.as_tensor(flags, dtype=torch.int32))
+            if rung is not None:
+                t.rung[:n].copy_(torch.as_tensor(rung, dtype=torch.int32))
+        t.n_chunks.fill_(n)
+        return t
+
+    def c_struct(self) -> CChunkTable:
+        return CChunkTable(_p(self.offsets), _p(self.rank), _p(self.scale), _p(self.rung), _p(self.flags),
+                           _p(self.n_chunks), self.capacity)
+
+    def to_host(self) -> dict:
+        n = int(self.n_chunks.item())
+        return dict(offsets=self.offsets[:n + 1].cpu().numpy(), rank=self.rank[:n].cpu().numpy(),
+                    scale=self.scale[:n].cpu().numpy(), rung=self.rung[:n].cpu().numpy(),
+                    flags=self.flags[:n].cpu().numpy(), n_chunks=n)
+
+
+def _check(call: str, status: int) -> None:
+    if status != 0:
+        raise CwlError(call, status)
+
+
+def cwl_score_tokens(logits: torch.Tensor, score: Optional[torch.Tensor] = None,
+                     stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """score[t] = normalised softmax entropy of logits[t, :] (fp32 [T, V] on the device)."""
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.dim() == 2 and logits.stride(1) == 1
+    T, V = logits.shape
+    if score is None:
+        score = torch.empty(T, dtype=torch.float32, device=logits.device)
+    _check("cwl_score_tokens", lib().cwl_score_tokens(_p(logits), logits.stride(0) if T > 1 else max(V, logits.stride(0)),
+                                                      T, V, _p(score), _stream_ptr(stream)))
+    return score
+
+
+def cwl_partition_workspace_bytes(T: int, n_seq: int) -> int:
+    return int(lib().cwl_partition_workspace_bytes(T, n_seq))
+
+
+def cwl_partition(score: torch.Tensor, cu_seqlens: torch.Tensor, policy: CPolicy,
+                  table: Optional[DeviceChunkTable] = None, workspace: Optional[torch.Tensor] = None,
+                  status_word: Optional[torch.Tensor] = None,
+                  stream: Optional[torch.cuda.Stream] = None) -> DeviceChunkTable:
+    """Adaptive chunker + rank-ladder selector; the table stays on the device."""
+    assert score.is_cuda and score.dtype == torch.float32 and score.is_contiguous()
+    assert cu_seqlens.is_cuda and cu_seqlens.dtype == torch.int32 and cu_seqlens.is_contiguous()
+    T, n_seq = score.shape[0], cu_seqlens.shape[0] - 1
+    if table is None:
+        table = DeviceChunkTable(T // max(int(policy.min_len), 1) + n_seq + 1, score.device)
+    need = cwl_partition_workspace_bytes(T, n_seq)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=score.device)
+    _check("cwl_partition", lib().cwl_partition(_p(score), _p(cu_seqlens), n_seq, T, C.byref(policy),
+                                                table.c_struct(), _p(workspace), workspace.numel(),
+                                                _p(status_word), _stream_ptr(stream)))
+    return table
+
+
+def cwl_apply_workspace_bytes(T: int, d_in: int, d_out: int, R: int) -> int:
+    return int(lib().cwl_apply_workspace_bytes(T, d_in, d_out, R))
+
+
+def cwl_apply(X: torch.Tensor, W: torch.Tensor, A: Optional[torch.Tensor], B: Optional[torch.Tensor],
+              table: Optional[DeviceChunkTable], window: int, Y: Optional[torch.Tensor] = None,
+              workspace: Optional[torch.Tensor] = None, status_word: Optional[torch.Tensor] = None,
+              stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Y = X W + gated (X A) B per the chunk table (bf16 tensors on the device, row-major)."""
+    for t in (X, W):
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.dim() == 2 and t.stride(1) == 1
+    T, d_in = X.shape
+    d_out = W.shape[1]
+    R = 0
+    if A is not None and B is not None:
+        assert A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16 and A.stride(1) == 1 and B.stride(1) == 1
+        R = A.shape[1]
+    if Y is None:
+        Y = torch.empty(T, d_out, dtype=torch.bfloat16, device=X.device)
+    need = cwl_apply_workspace_bytes(T, d_in, d_out, R)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=X.device)
+    ct = table.c_struct() if table is not None else CChunkTable(None, None, None, None, None, None, 0)
+    _check("cwl_apply", lib().cwl_apply(_p(X), X.stride(0), _p(W), W.stride(0),
+                                        _p(A), A.stride(0) if R else 0, _p(B), B.stride(0) if R else 0,
+                                        T, d_in, d_out, R, ct, int(window), _p(Y), Y.stride(0),
+                                        _p(workspace), workspace.numel(), _p(status_word), _stream_ptr(stream)))
+    return Y
+
+
+def bf16_from_bits(bits, device="cuda") -> torch.Tensor:
+    """uint16 bit patterns (numpy) -> bf16 tensor on the device, no rounding involved."""
+    import numpy as np
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16))
+    return t.to(device).view(torch.bfloat16)

@@ -1,0 +1,346 @@
+// cwl_partition: adaptive chunker (Sec. III-B) and rank-ladder selector (Sec. III-C).
+//
+// The greedy walk is chunk-sequential, but the cut that follows a chunk start b depends on b
+// alone.  So the work is split into data-parallel passes and one short pointer chase:
+//   1. quantise scores to Q24 integers and reduce per tile            (grid over T)
+//   2. exclusive prefix sums P[0..T] (int64)                          (grid over T)
+//   3. next_cut[b] for EVERY position b: first stopping candidate     (one warp per b, ballot)
+//   4. per sequence: chase next_cut from the sequence start through shared memory, then
+//      rung per chunk and the high-capacity budget                    (one block per sequence)
+//   5. compact the per-sequence lists into the caller's chunk table   (one block per sequence)
+// All comparisons are integer, so the table is a function of the fp32 scores only.
+#include "cwl_common.cuh"
+
+namespace cwl {
+namespace {
+
+constexpr int kScanThreads = 256;
+constexpr int kScanItems = 8;
+constexpr int kScanTile = kScanThreads * kScanItems;  // scores per block in passes 1 and 2
+constexpr int kWalkThreads = 256;
+constexpr int kWalkSegment = 8192;                    // next_cut entries staged per shared-memory segment
+
+struct Ladder {
+  int32_t n_rungs;
+  int32_t min_len, max_len, hi_budget;
+  int64_t theta_q[CWL_MAX_RUNGS - 1];  // floor(threshold * 2^24)
+  int32_t rung_rank[CWL_MAX_RUNGS];
+  float rung_scale[CWL_MAX_RUNGS];
+};
+
+struct Workspace {
+  int64_t* P;          // [T + 1]
+  int64_t* tile_sum;   // [n_tiles]
+  int32_t* next_cut;   // [T]
+  int32_t* seq_start;  // [T] chunk starts of sequence n live at [cu[n], cu[n] + count[n])
+  int32_t* seq_rung0;  // [T] rung as walked
+  int32_t* seq_rung;   // [T] rung after the budget
+  int32_t* count;      // [n_seq]
+};
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+inline size_t carve(Workspace& w, char* base, int32_t T, int32_t n_seq) {
+  size_t off = 0;
+  const size_t n_tiles = (size_t)ceil_div64(T > 0 ? T : 1, kScanTile);
+  auto take = [&](size_t bytes) { char* p = base ? base + off : nullptr; off = align_up(off + bytes, 16); return p; };
+  w.P = reinterpret_cast<int64_t*>(take(sizeof(int64_t) * ((size_t)T + 1)));
+  w.tile_sum = reinterpret_cast<int64_t*>(take(sizeof(int64_t) * n_tiles));
+  w.next_cut = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * (size_t)(T > 0 ? T : 1)));
+  w.seq_start = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * (size_t)(T > 0 ? T : 1)));
+  w.seq_rung0 = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * (size_t)(T > 0 ? T : 1)));
+  w.seq_rung = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * (size_t)(T > 0 ? T : 1)));
+  w.count = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * (size_t)(n_seq > 0 ? n_seq : 1)));
+  return off;
+}
+
+__device__ __forceinline__ int32_t quantise(float s) {
+  if (s != s) return kQ24;  // NaN: hardest
+  s = fminf(fmaxf(s, 0.f), 1.f);
+  return __float2int_rd(s * 16777216.0f);  // exact: power-of-two scaling, then floor
+}
+
+__device__ __forceinline__ int rung_of(int64_t sum, int64_t len, const Ladder& L) {
+  int k = 0;
+#pragma unroll
+  for (int j = 0; j < CWL_MAX_RUNGS - 1; ++j)
+    if (j + 1 < L.n_rungs && sum >= L.theta_q[j] * len) ++k;
+  return k;
+}
+
+__device__ __forceinline__ int64_t warp_sum64(int64_t v) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+  return v;
+}
+
+// Block-wide sum of one int64 per thread; result valid in every thread.
+__device__ int64_t block_sum64(int64_t v, int64_t* smem /* >= 32 entries */) {
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  v = warp_sum64(v);
+  __syncthreads();
+  if (lane == 0) smem[wid] = v;
+  __syncthreads();
+  int64_t t = (lane < nw) ? smem[lane] : 0;
+  return warp_sum64(t);
+}
+
+// pass 1: per-tile sums of quantised scores
+__global__ void __launch_bounds__(kScanThreads)
+tile_sum_kernel(const float* __restrict__ score, int T, int64_t* __restrict__ tile_sum) {
+  __shared__ int64_t red[32];
+  const int base = blockIdx.x * kScanTile;
+  int64_t s = 0;
+#pragma unroll
+  for (int i = 0; i < kScanItems; ++i) {
+    int t = base + i * kScanThreads + threadIdx.x;
+    if (t < T) s += quantise(score[t]);
+  }
+  s = block_sum64(s, red);
+  if (threadIdx.x == 0) tile_sum[blockIdx.x] = s;
+}
+
+// pass 2: exclusive prefix sums.  Each block adds up the tiles before it, then scans its own.
+__global__ void __launch_bounds__(kScanThreads)
+prefix_kernel(const float* __restrict__ score, int T, const int64_t* __restrict__ tile_sum,
+              int64_t* __restrict__ P) {
+  __shared__ int64_t red[32];
+  __shared__ int64_t warp_tot[kScanThreads / 32];
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  int64_t before = 0;
+  for (int i = tid; i < (int)blockIdx.x; i += kScanThreads) before += tile_sum[i];
+  before = block_sum64(before, red);
+
+  // thread-contiguous items: thread tid owns [base + tid*kScanItems, +kScanItems)
+  const int t0 = blockIdx.x * kScanTile + tid * kScanItems;
+  int32_t q[kScanItems];
+  int64_t mine = 0;
+#pragma unroll
+  for (int i = 0; i < kScanItems; ++i) {
+    q[i] = (t0 + i < T) ? quantise(score[t0 + i]) : 0;
+    mine += q[i];
+  }
+  int64_t incl = mine;  // inclusive warp scan of per-thread totals
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    int64_t o = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += o;
+  }
+  if (lane == 31) warp_tot[wid] = incl;
+  __syncthreads();
+  int64_t warp_before = 0;
+  for (int w = 0; w < wid; ++w) warp_before += warp_tot[w];
+  int64_t run = before + warp_before + (incl - mine);
+#pragma unroll
+  for (int i = 0; i < kScanItems; ++i) {
+    if (t0 + i < T) P[t0 + i] = run;
+    run += q[i];
+    if (t0 + i == T - 1) P[T] = run;
+  }
+  if (T == 0 && blockIdx.x == 0 && tid == 0) P[0] = 0;
+}
+
+// pass 3: the cut that closes a chunk opened at b (one warp per b)
+__global__ void __launch_bounds__(256)
+next_cut_kernel(const int64_t* __restrict__ P, const int32_t* __restrict__ cu, int n_seq, int T,
+                Ladder L, int32_t* __restrict__ next_cut) {
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  for (int64_t b64 = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); b64 < T;
+       b64 += (int64_t)gridDim.x * warps_per_block) {
+    const int b = (int)b64;
+    // sequence of b: last n with cu[n] <= b (skips empty sequences)
+    int lo = 0, hi = n_seq;  // invariant: cu[lo] <= b < cu[hi]
+    while (hi - lo > 1) {
+      int mid = (lo + hi) >> 1;
+      if (cu[mid] <= b) lo = mid; else hi = mid;
+    }
+    const int E = cu[lo + 1];
+    int cut = E;
+    if (E - b >= 2 * L.min_len) {
+      const int first = b + L.min_len;
+      const int last = min(E - L.min_len, b + L.max_len);  // the candidate at b + max_len always stops
+      const int64_t Pb = P[b];
+      for (int base = first; base <= last; base += 32) {
+        const int e = base + lane;
+        bool stop = false;
+        if (e <= last) {
+          if (e - b >= L.max_len) {
+            stop = true;
+          } else {
+            const int64_t Pe = P[e];
+            stop = rung_of(Pe - Pb, e - b, L) != rung_of(P[e + L.min_len] - Pe, L.min_len, L);
+          }
+        }
+        const unsigned m = __ballot_sync(0xffffffffu, stop);
+        if (m) { cut = base + __ffs(m) - 1; break; }
+      }
+    }
+    if (lane == 0) next_cut[b] = cut;
+  }
+}
+
+// pass 4: chase the cuts of one sequence, then rung and budget per chunk
+__global__ void __launch_bounds__(kWalkThreads)
+walk_kernel(const int64_t* __restrict__ P, const int32_t* __restrict__ cu, Ladder L,
+            const int32_t* __restrict__ next_cut, int32_t* __restrict__ seq_start,
+            int32_t* __restrict__ seq_rung0, int32_t* __restrict__ seq_rung, int32_t* __restrict__ count) {
+  __shared__ int32_t seg[kWalkSegment];
+  __shared__ int s_pos, s_count;
+  const int n = blockIdx.x, tid = threadIdx.x;
+  const int S = cu[n], E = cu[n + 1];
+  if (tid == 0) { s_pos = S; s_count = 0; }
+  __syncthreads();
+  while (true) {
+    const int seg_base = s_pos;
+    if (seg_base >= E) break;
+    const int seg_end = min(E, seg_base + kWalkSegment);
+    for (int i = seg_base + tid; i < seg_end; i += kWalkThreads) seg[i - seg_base] = next_cut[i];
+    __syncthreads();
+    if (tid == 0) {
+      int b = seg_base, c = s_count;
+      while (b < seg_end) {
+        seq_start[S + c] = b;   // chunks are non-empty, so a sequence never has more chunks than tokens
+        ++c;
+        b = seg[b - seg_base];
+      }
+      s_pos = b;
+      s_count = c;
+    }
+    __syncthreads();
+  }
+  const int C = s_count;
+  if (tid == 0) count[n] = C;
+  // rung of every chunk as walked
+  for (int c = tid; c < C; c += kWalkThreads) {
+    const int b = seq_start[S + c], e = (c + 1 < C) ? seq_start[S + c + 1] : E;
+    const int r = rung_of(P[e] - P[b], e - b, L);
+    seq_rung0[S + c] = r;
+    seq_rung[S + c] = r;
+  }
+  if (L.hi_budget < 0 || L.n_rungs < 2) return;
+  __syncthreads();
+  // budget on high-capacity regions: a top-rung chunk keeps its rung only if fewer than
+  // hi_budget top-rung chunks of this sequence have a larger mean (earlier chunk wins ties)
+  const int top = L.n_rungs - 1;
+  for (int c = tid; c < C; c += kWalkThreads) {
+    if (seq_rung0[S + c] != top) continue;
+    const int bc = seq_start[S + c], ec = (c + 1 < C) ? seq_start[S + c + 1] : E;
+    const int64_t sum_c = P[ec] - P[bc], len_c = ec - bc;
+    int better = 0;
+    for (int d = 0; d < C; ++d) {
+      if (d == c || seq_rung0[S + d] != top) continue;
+      const int bd = seq_start[S + d], ed = (d + 1 < C) ? seq_start[S + d + 1] : E;
+      const int64_t lhs = (P[ed] - P[bd]) * len_c, rhs = sum_c * (int64_t)(ed - bd);
+      if (lhs > rhs || (lhs == rhs && d < c)) ++better;
+    }
+    if (better >= L.hi_budget) seq_rung[S + c] = top - 1;
+  }
+}
+
+// pass 5: compaction into the caller's table
+__global__ void __launch_bounds__(256)
+emit_kernel(const int32_t* __restrict__ cu, int n_seq, int T, Ladder L,
+            const int32_t* __restrict__ seq_start, const int32_t* __restrict__ seq_rung,
+            const int32_t* __restrict__ count, cwl_chunk_table table, int32_t* status_word) {
+  __shared__ int64_t red[32];
+  const int n = blockIdx.x, tid = threadIdx.x;
+  int64_t before = 0;
+  for (int i = tid; i < n && i < n_seq; i += blockDim.x) before += count[i];
+  const int base = (int)block_sum64(before, red);
+  const int C = (n < n_seq) ? count[n] : 0;
+  const bool fits = (int64_t)base + C <= (int64_t)table.capacity;
+  if (n < n_seq && fits) {
+    const int S = cu[n];
+    for (int c = tid; c < C; c += blockDim.x) {
+      const int r = seq_rung[S + c];
+      table.offsets[base + c] = seq_start[S + c];
+      table.rung[base + c] = r;
+      table.rank[base + c] = L.rung_rank[r];
+      table.scale[base + c] = L.rung_scale[r];
+      table.flags[base + c] = (c == 0) ? 1 : 0;
+    }
+  }
+  if (n == max(n_seq, 1) - 1 && tid == 0) {  // the last block owns the totals
+    if (fits) {
+      table.offsets[base + C] = T;
+      *table.n_chunks = base + C;
+    } else {
+      *table.n_chunks = 0;
+      flag_status(status_word, CWL_ERR_CAPACITY);
+    }
+  }
+}
+
+bool policy_ok(const cwl_policy* p) {
+  if (p == nullptr || p->n_rungs < 1 || p->n_rungs > CWL_MAX_RUNGS) return false;
+  if (p->min_len < 1 || p->max_len < p->min_len) return false;
+  if ((int64_t)p->min_len + (int64_t)p->max_len > (int64_t)(1 << 19)) return false;
+  if (p->window < 0 || p->window > p->min_len) return false;
+  for (int k = 0; k < p->n_rungs; ++k) {
+    if (p->rung_rank[k] < 0 || p->rung_rank[k] > CWL_MAX_RANK) return false;
+    if (k > 0 && p->rung_rank[k] < p->rung_rank[k - 1]) return false;
+  }
+  for (int k = 0; k + 1 < p->n_rungs; ++k) {
+    const float th = p->threshold[k];
+    if (!(th >= 0.f && th <= 1.f)) return false;
+    if (k > 0 && !(th > p->threshold[k - 1])) return false;
+  }
+  return true;
+}
+
+}  // namespace
+}  // namespace cwl
+
+extern "C" size_t cwl_partition_workspace_bytes(int32_t T, int32_t n_seq) {
+  if (T < 0 || n_seq < 0) return 0;
+  cwl::Workspace w;
+  return cwl::carve(w, nullptr, T, n_seq);
+}
+
+extern "C" cwl_status cwl_partition(const float* score, const int32_t* cu_seqlens, int32_t n_seq, int32_t T,
+                                    const cwl_policy* policy, cwl_chunk_table table,
+                                    void* workspace, size_t workspace_bytes,
+                                    int32_t* status_word, void* stream_) {
+  using namespace cwl;
+  if (T < 0 || n_seq < 0 || cu_seqlens == nullptr || (score == nullptr && T > 0)) return CWL_ERR_INVALID_ARG;
+  if (!policy_ok(policy)) return CWL_ERR_INVALID_ARG;
+  if (table.offsets == nullptr || table.rank == nullptr || table.scale == nullptr || table.rung == nullptr ||
+      table.flags == nullptr || table.n_chunks == nullptr || table.capacity < 0)
+    return CWL_ERR_INVALID_ARG;
+  if (T > 0 && n_seq == 0) return CWL_ERR_INVALID_ARG;
+  Workspace w;
+  const size_t need = carve(w, static_cast<char*>(workspace), T, n_seq);
+  if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return CWL_ERR_WORKSPACE;
+
+  Ladder L{};
+  L.n_rungs = policy->n_rungs;
+  L.min_len = policy->min_len;
+  L.max_len = policy->max_len;
+  L.hi_budget = policy->hi_budget;
+  for (int k = 0; k < policy->n_rungs; ++k) {
+    L.rung_rank[k] = policy->rung_rank[k];
+    L.rung_scale[k] = policy->rung_scale[k];
+  }
+  for (int k = 0; k + 1 < policy->n_rungs; ++k)
+    L.theta_q[k] = (int64_t)__builtin_floor((double)policy->threshold[k] * 16777216.0);
+
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (T > 0) {
+    const int n_tiles = (int)ceil_div64(T, kScanTile);
+    tile_sum_kernel<<<n_tiles, kScanThreads, 0, stream>>>(score, T, w.tile_sum);
+    prefix_kernel<<<n_tiles, kScanThreads, 0, stream>>>(score, T, w.tile_sum, w.P);
+    const int warps_per_block = 8;
+    int64_t blocks = ceil_div64(T, warps_per_block);
+    if (blocks > 148 * 64) blocks = 148 * 64;
+    next_cut_kernel<<<(int)blocks, warps_per_block * 32, 0, stream>>>(w.P, cu_seqlens, n_seq, T, L, w.next_cut);
+    walk_kernel<<<n_seq, kWalkThreads, 0, stream>>>(w.P, cu_seqlens, L, w.next_cut, w.seq_start,
+                                                   w.seq_rung0, w.seq_rung, w.count);
+  } else if (n_seq > 0) {
+    CWL_CUDA_TRY(cudaMemsetAsync(w.count, 0, sizeof(int32_t) * (size_t)n_seq, stream));
+  }
+  emit_kernel<<<n_seq > 0 ? n_seq : 1, 256, 0, stream>>>(cu_seqlens, n_seq, T, L, w.seq_start, w.seq_rung,
+                                                         w.count, table, status_word);
+  CWL_CUDA_TRY(cudaGetLastError());
+  return CWL_OK;
+}
