@@ -1,0 +1,404 @@
+#!/usr/bin/env python
+"""Benchmark of the ChunkWise-LoRA hot path on B200.
+
+One step = one pass of the whole hot path over one batch of the LLaMA-7B-shaped prefill
+configuration (T = 2048 tokens): token scoring from fp32 logits [T, 32000], adaptive partition and
+rank selection, then the adapted projection for all seven projections (q, k, v, o, gate, up, down)
+with R = 64.  Prints ONE JSON line (see README for the fields).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg2|cfg4|cfg1]
+
+N > 1 runs N independent replicas (one process per GPU, launched with torch.distributed.run); the
+path has no exchange step, so there is no data-path collective: only the timing barrier and the
+max-over-ranks reduction of the timed region.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "adapted_projection_tokens_per_s"
+UNIT = "tokens/s"
+
+
+# ------------------------------------------------------------------------------------ helpers
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def load_traffic(kernel: str):
+    """DRAM bytes per launch of the dominant kernel from a committed ncu summary, or None."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as fh:
+        return json.load(fh).get(kernel)
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        inside = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.1] or [l for (_, l) in self.lines]
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in inside:
+            parts = [x.strip() for x in l.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def table_flops(table: dict, window: int, T: int, projs, R: int):
+    """Algorithmic and executed FLOPs of the adapted projections for one step."""
+    off, rank, flags = table["offsets"], table["rank"], table["flags"]
+    active = np.zeros(T, dtype=np.int64)
+    for c in range(table["n_chunks"]):
+        active[off[c]:off[c + 1]] = rank[c]
+        if c > 0 and not (flags[c] & 1):
+            w = min(window, off[c + 1] - off[c])
+            active[off[c]:off[c] + w] = max(rank[c], rank[c - 1])
+    rsum = int(active.sum())
+    alg = sum(2 * T * d_in * d_out + 2 * rsum * (d_in + d_out) for (d_in, d_out) in projs)
+    exe = sum(2 * T * d_in * d_out + 2 * T * R * (d_in + d_out) for (d_in, d_out) in projs)
+    return alg, exe
+
+
+def make_workload(name: str):
+    from paper_2601_21109_b200 import workloads as wl
+    if name == "cfg2":
+        return wl.config2()
+    if name == "cfg1":
+        return wl.config1()
+    if name == "cfg4":
+        return wl.config4()
+    raise SystemExit(f"unknown workload {name}")
+
+
+# ----------------------------------------------------------------------------- reference arm
+def oracle_sample(w, n_rows: int, n_score_rows: int = 64):
+    """Times the fp64 CPU oracle on a bounded sample of the workload; returns (tokens/s, info)."""
+    import oracle
+    cores = oracle.get_threads()
+    p = w.policy
+    rng = np.random.default_rng(0)
+    t0 = time.perf_counter()
+    if w.logits is not None:
+        srows = np.sort(rng.choice(w.T, size=min(w.T, n_score_rows), replace=False))
+        s_sample = oracle.score_tokens(w.logits[srows])
+        t_score = (time.perf_counter() - t0) * (w.T / len(srows))          # scaled to all T rows
+        score = np.interp(np.arange(w.T), srows, s_sample).astype(np.float32)  # stand-in track for the partition timing
+        ths = np.percentile(s_sample, [25, 50, 75]).astype(np.float32).tolist()
+    else:
+        srows, t_score, score, ths = [], 0.0, w.score, p.thresholds
+    t1 = time.perf_counter()
+    if w.table is None:
+        tab = oracle.partition(score, w.cu_seqlens, p.ranks, p.scales, ths, p.min_len, p.max_len, p.window, p.hi_budget)
+    else:
+        t = w.table
+        tab = oracle.ChunkTable(t["offsets"], t["rank"], t["scale"], t["rung"], t["flags"], t["n_chunks"])
+    t_part = time.perf_counter() - t1
+    rows = np.sort(rng.choice(w.T, size=min(n_rows, w.T), replace=False)).astype(np.int32)
+    t2 = time.perf_counter()
+    for pr in w.projections:
+        oracle.apply(w.X[pr.d_in], pr.W, pr.A, pr.B, tab, p.window, rows=rows)
+    t_apply_sample = time.perf_counter() - t2
+    t_apply = t_apply_sample * (w.T / len(rows))                            # per-row cost is constant
+    total = t_score + t_part + t_apply
+    info = dict(cores=cores, kind="oracle",
+                sample=f"{len(rows)} of {w.T} rows through all {len(w.projections)} projections (fp64 naive loops), "
+                       f"score on {len(srows)} rows, partition in full; times scaled to {w.T} rows",
+                sample_seconds=time.perf_counter() - t0)
+    return w.T / total, info
+
+
+def rows_for_budget(w, seconds: float):
+    """Sample size whose oracle run takes about `seconds` on this host (calibrated on one row per core)."""
+    import oracle
+    cores = oracle.get_threads()
+    t0 = time.perf_counter()
+    oracle_sample(w, n_rows=cores, n_score_rows=8)
+    t_wave = max(time.perf_counter() - t0, 1e-3)      # one row per core through every projection
+    waves = max(1, int(seconds / t_wave))
+    return int(min(w.T, cores * waves)), t_wave
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = make_workload(args.workload)
+    budget = 150.0 / (args.steps + args.warmup)         # the whole run ends within a few minutes
+    n_rows, _ = rows_for_budget(w, budget)
+    vals = []
+    info = {}
+    for i in range(args.warmup + args.steps):
+        v, info = oracle_sample(w, n_rows)
+        if i >= args.warmup:
+            vals.append(v)
+    value = float(np.mean(vals))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.T / value,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "T": w.T, "R": w.R, "projections": [f"{p.name}:{p.d_in}x{p.d_out}" for p in w.projections]},
+            "cpu_baseline": dict(value=value, unit=UNIT, **info),
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2601_21109_b200 import binding as cwl
+    from paper_2601_21109_b200.runner import HotPath
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    cwl.lib()  # fails loudly when libcwl.so is missing
+
+    w = make_workload(args.workload)
+    hp = HotPath(w)
+    stream = torch.cuda.current_stream()
+
+    # thresholds of the rule-based percentile mapping (Sec. IV-C): quartiles of this batch's scores
+    if hp.logits is not None:
+        hp.score_step()
+        s = hp.score.cpu().numpy()
+        hp.set_thresholds(np.percentile(s, [25, 50, 75]).astype(np.float32).tolist())
+    hp.step()
+    torch.cuda.synchronize()
+    if int(hp.status.item()) != 0:
+        raise SystemExit(f"device status word {int(hp.status.item()):#x}")
+    table = hp.table.to_host()
+    proj_dims = [(p.d_in, p.d_out) for p in hp.projs]
+    f_alg, f_exe = table_flops(table, hp.policy.window, hp.T, proj_dims, hp.R)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing --------------------------------------------------------------
+    for _ in range(args.warmup):
+        hp.step()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    barrier()
+    t_wall0 = time.time()
+    e0.record(stream)
+    for i in range(args.steps):
+        if hp.logits is not None:
+            hp.score_step()
+        if not hp.fixed_table:
+            hp.partition_step()
+        ev[i][0].record(stream)
+        hp.apply_step()
+        ev[i][1].record(stream)
+    e1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    ms_total = e0.elapsed_time(e1)
+    apply_ms = [a.elapsed_time(b) for a, b in ev]
+    if world > 1:
+        t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    if int(hp.status.item()) != 0:
+        raise SystemExit(f"device status word {int(hp.status.item()):#x}")
+    tokens_total = hp.T * args.steps * world
+    value = tokens_total / (ms_total * 1e-3)
+
+    # ---- comparison runs through the same kernels: static full-rank LoRA and the dense floor ---
+    from paper_2601_21109_b200 import workloads as wl
+    st = wl.static_table(w.cu_seqlens, hp.R, 32.0)
+    static_tab = cwl.DeviceChunkTable.from_host(st["offsets"], st["rank"], st["scale"], st["flags"], st["rung"])
+
+    def time_apply(**kw):
+        for _ in range(3):
+            hp.apply_step(**kw)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = max(5, min(args.steps, 50))
+        a.record(stream)
+        for _ in range(n):
+            hp.apply_step(**kw)
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+    static_ms = time_apply(table=static_tab)
+    dense_ms = time_apply(dense=True)
+
+    # ---- end to end: pinned host inputs in, results out, every step ----------------------------
+    host_in = {d: x.cpu().pin_memory() for d, x in hp.X.items()}
+    host_logits = hp.logits.cpu().pin_memory() if hp.logits is not None else None
+    host_out = [torch.empty(p.Y.shape, dtype=p.Y.dtype).pin_memory() for p in hp.projs]
+    h2d = sum(x.numel() * x.element_size() for x in host_in.values()) + \
+        (host_logits.numel() * 4 if host_logits is not None else 0)
+    d2h = sum(y.numel() * y.element_size() for y in host_out)
+    e2e_steps = max(3, min(args.steps, 20))
+
+    def e2e_step():
+        for d, x in host_in.items():
+            hp.X[d].copy_(x, non_blocking=True)
+        if host_logits is not None:
+            hp.logits.copy_(host_logits, non_blocking=True)
+        hp.step()
+        for p, y in zip(hp.projs, host_out):
+            y.copy_(p.Y, non_blocking=True)
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    b.record(stream)
+    barrier()
+    e2e_ms = a.elapsed_time(b)
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = hp.T * e2e_steps * world / (e2e_ms * 1e-3)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (the projection GEMM inside cwl_apply) -----------------
+    peaks = load_peaks()
+    apply_avg_ms = float(np.mean(apply_ms))
+    region_s = ms_total * 1e-3
+    if args.workload == "cfg4":
+        bytes_alg = sum(2 * (hp.T * di + di * do + hp.R * (di + do) + hp.T * do) + 2 * hp.T * hp.R * 2 for di, do in proj_dims)
+        achieved = bytes_alg / (apply_avg_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": load_traffic("apply_" + args.workload),
+                "peak_source": f"hbm copy, of {peaks['source']}"}
+    else:
+        kind = "bf16_tflops_sustained" if region_s > 1.0 else "bf16_tflops"
+        achieved = f_alg / (apply_avg_ms * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks[kind], "unit": "TFLOP/s",
+                "frac": achieved / peaks[kind], "traffic": load_traffic("apply_" + args.workload),
+                "peak_source": f"{kind}, of {peaks['source']}"}
+    roof["kernel"] = "cwl_apply (shrink + gate + projection GEMM; the event bracket spans all launches of the 7 applies of a step)"
+    roof["launch_ms"] = apply_avg_ms
+    roof["executed_tflops"] = f_exe / (apply_avg_ms * 1e-3) / 1e12
+    roof["frac_of_nominal_2250"] = (f_alg / (apply_avg_ms * 1e-3) / 1e12) / 2250.0
+
+    n_rows, _ = rows_for_budget(w, 12.0)             # about 10-20 s of CPU work
+    cpu_val, cpu_info = oracle_sample(w, n_rows=n_rows)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "T": hp.T, "R": hp.R, "projections": [f"{p.name}:{p.d_in}x{p.d_out}" for p in hp.projs],
+                   "ladder": hp.policy.ranks, "window": hp.policy.window, "min_len": hp.policy.min_len,
+                   "n_chunks": table["n_chunks"], "steps_include": "score + partition + 7 x apply",
+                   "l2": "inputs larger than L2 (400 MB of weights + 262 MB of logits per step)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "tflops": f_alg * args.steps * world / (ms_total * 1e-3) / 1e12,
+        "apply_ms_per_step": apply_avg_ms,
+        "static_lora_apply_ms": static_ms, "dense_floor_apply_ms": dense_ms,
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": hp.launches_per_step() * args.steps,
+        "roofline": roof,
+        "cpu_baseline": dict(value=cpu_val, unit=UNIT, **cpu_info),
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg4"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 2 if args.steps is None else max(1, args.steps)
+        args.warmup = 1 if args.warmup is None else max(0, args.warmup)
+        run_reference(args)
+    else:
+        args.steps = 200 if args.steps is None else max(1, args.steps)
+        args.warmup = max(5 if args.warmup is None else args.warmup, 3)
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -560,8 +560,9 @@ extern "C" cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64
                                 void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
                                 int32_t* status_word, void* stream_) {
   using namespace cwl;
-  if (X == nullptr || W == nullptr || Y == nullptr || T < 0 || d_in < 1 || d_out < 1 || R < 0 || window < 0)
-    return CWL_ERR_INVALID_ARG;
+  if (T < 0 || d_in < 1 || d_out < 1 || R < 0 || window < 0) return CWL_ERR_INVALID_ARG;
+  if (T > 0 && (X == nullptr || Y == nullptr)) return CWL_ERR_INVALID_ARG;
+  if (W == nullptr) return CWL_ERR_INVALID_ARG;
   const bool adapter = (A != nullptr && B != nullptr && R > 0);
   if (d_in % 16 != 0 || d_out % 16 != 0) return CWL_ERR_UNSUPPORTED;
   if (adapter && (R % 16 != 0 || R > CWL_MAX_RANK)) return CWL_ERR_UNSUPPORTED;
@@ -569,10 +570,10 @@ extern "C" cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64
   if (ldx % 8 != 0 || ldw % 8 != 0 || ldy % 8 != 0 || (adapter && (lda % 8 != 0 || ldb % 8 != 0))) return CWL_ERR_SHAPE;
   if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || (adapter && (!aligned16(A) || !aligned16(B))))
     return CWL_ERR_SHAPE;
+  if (T == 0) return CWL_OK;
   if (adapter && (table.offsets == nullptr || table.rank == nullptr || table.scale == nullptr ||
                   table.flags == nullptr || table.n_chunks == nullptr || table.capacity < 0))
     return CWL_ERR_INVALID_ARG;
-  if (T == 0) return CWL_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
 
   ApplyWorkspace ws{nullptr, nullptr};

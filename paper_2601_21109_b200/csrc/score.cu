@@ -35,9 +35,9 @@ __device__ __forceinline__ void rebase(Triple& a, float m_new) {
   a.m = m_new;
 }
 
-__device__ __forceinline__ void absorb(Triple& a, float z, float neg_m_l2e) {
-  float t = fmaf(z, kLog2e, neg_m_l2e);
-  t = fmaxf(t, -1.0e30f);                 // z = -inf: weight 0 and product 0 instead of NaN
+__device__ __forceinline__ void absorb(Triple& a, float z, float m) {
+  // z - m first (exact when z == m, even for huge |m|), then into the log2 domain
+  float t = fmaxf((z - m) * kLog2e, -1.0e30f);  // z = -inf: weight 0 and product 0 instead of NaN
   float e = ex2_approx(t);
   a.S += e;
   a.U = fmaf(t, e, a.U);
@@ -76,7 +76,7 @@ score_rows_kernel(const float* __restrict__ logits, int64_t ld, int T, int V, fl
       float m_new = fmaxf(acc.m, v);
       if (m_new == -CUDART_INF_F) return;
       if (m_new > acc.m) rebase(acc, m_new);
-      absorb(acc, v, -acc.m * kLog2e);
+      absorb(acc, v, acc.m);
     };
     if (tid < head) take_scalar(z[tid]);
     if (tid < V - tail_start) take_scalar(z[tail_start + tid]);
@@ -90,11 +90,11 @@ score_rows_kernel(const float* __restrict__ logits, int64_t ld, int T, int V, fl
       float m_new = fmaxf(acc.m, m4);
       if (m_new == -CUDART_INF_F) continue;
       if (m_new > acc.m) rebase(acc, m_new);
-      const float nm = -acc.m * kLog2e;
-      absorb(acc, v.x, nm);
-      absorb(acc, v.y, nm);
-      absorb(acc, v.z, nm);
-      absorb(acc, v.w, nm);
+      const float m = acc.m;
+      absorb(acc, v.x, m);
+      absorb(acc, v.y, m);
+      absorb(acc, v.z, m);
+      absorb(acc, v.w, m);
     }
 
     int bad = ok ? 0 : 1;
@@ -142,10 +142,11 @@ score_rows_kernel(const float* __restrict__ logits, int64_t ld, int T, int V, fl
 
 extern "C" cwl_status cwl_score_tokens(const float* logits, int64_t ld_logits, int32_t T, int32_t V,
                                        float* score, void* stream) {
-  if (logits == nullptr || score == nullptr || T < 0 || V < 2) return CWL_ERR_INVALID_ARG;
+  if (T < 0 || V < 2) return CWL_ERR_INVALID_ARG;
+  if (T == 0) return CWL_OK;
+  if (logits == nullptr || score == nullptr) return CWL_ERR_INVALID_ARG;
   if (ld_logits < V) return CWL_ERR_SHAPE;
   if ((reinterpret_cast<uintptr_t>(logits) & 3u) != 0) return CWL_ERR_SHAPE;
-  if (T == 0) return CWL_OK;
   int grid = T < (1 << 20) ? T : (1 << 20);
   cwl::score_rows_kernel<<<grid, cwl::kScoreThreads, 0, static_cast<cudaStream_t>(stream)>>>(
       logits, ld_logits, T, V, score);

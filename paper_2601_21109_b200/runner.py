@@ -1,0 +1,101 @@
+"""Orchestration of one pass of the hot path over a batch: which C calls, in which order.
+
+``HotPath`` keeps the model state resident on the device (weights, adapter factors, workspaces,
+the chunk table) and issues score -> partition -> apply for every projection on one stream.  It
+contains no arithmetic of the method: thresholds, ladders and windows are handed to the library
+as they are.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Dict, List, Optional
+
+import numpy as np
+import torch
+
+from . import binding as cwl
+from .workloads import Policy, Workload
+
+
+@dataclass
+class DeviceProjection:
+    name: str
+    d_in: int
+    d_out: int
+    W: torch.Tensor
+    A: torch.Tensor
+    B: torch.Tensor
+    Y: torch.Tensor
+
+
+def policy_struct(p: Policy) -> cwl.CPolicy:
+    return cwl.make_policy(p.ranks, p.scales, p.thresholds, p.min_len, p.max_len, p.window, p.hi_budget)
+
+
+class HotPath:
+    """Device-resident state of one layer's adapted projections plus the scheduler in front."""
+
+    def __init__(self, w: Workload, device: str = "cuda", keep_host: bool = False):
+        self.T, self.R, self.policy = w.T, w.R, w.policy
+        self.device = device
+        self.cu_seqlens = torch.from_numpy(w.cu_seqlens).to(device)
+        self.n_seq = int(w.cu_seqlens.shape[0] - 1)
+        self.X: Dict[int, torch.Tensor] = {d: cwl.bf16_from_bits(x, device) for d, x in w.X.items()}
+        self.logits = torch.from_numpy(w.logits).to(device) if w.logits is not None else None
+        self.score = (torch.from_numpy(w.score).to(device) if w.score is not None
+                      else torch.empty(w.T, dtype=torch.float32, device=device))
+        self.projs: List[DeviceProjection] = []
+        for p in w.projections:
+            self.projs.append(DeviceProjection(
+                p.name, p.d_in, p.d_out, cwl.bf16_from_bits(p.W, device), cwl.bf16_from_bits(p.A, device),
+                cwl.bf16_from_bits(p.B, device), torch.empty(w.T, p.d_out, dtype=torch.bfloat16, device=device)))
+        cap = w.T // max(w.policy.min_len, 1) + self.n_seq + 1
+        self.table = cwl.DeviceChunkTable(cap, device)
+        if w.table is not None:
+            t = w.table
+            self.table = cwl.DeviceChunkTable.from_host(t["offsets"], t["rank"], t["scale"], t["flags"], t.get("rung"), device)
+        self.fixed_table = w.table is not None
+        self.part_ws = torch.empty(cwl.cwl_partition_workspace_bytes(w.T, self.n_seq), dtype=torch.uint8, device=device)
+        ws_bytes = max(cwl.cwl_apply_workspace_bytes(w.T, p.d_in, p.d_out, w.R) for p in w.projections)
+        self.apply_ws = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.cpolicy = policy_struct(w.policy)
+
+    # launches per call, for the benchmark's kernel count
+    LAUNCHES_SCORE = 1
+    LAUNCHES_PARTITION = 5
+    LAUNCHES_APPLY = 3
+    LAUNCHES_APPLY_DENSE = 1
+
+    def set_thresholds(self, thresholds) -> None:
+        self.policy.thresholds = [float(np.float32(t)) for t in thresholds]
+        self.cpolicy = policy_struct(self.policy)
+
+    def score_step(self) -> None:
+        cwl.cwl_score_tokens(self.logits, self.score)
+
+    def partition_step(self) -> None:
+        cwl.cwl_partition(self.score, self.cu_seqlens, self.cpolicy, table=self.table, workspace=self.part_ws,
+                          status_word=self.status)
+
+    def apply_step(self, table: Optional[cwl.DeviceChunkTable] = None, dense: bool = False) -> None:
+        tab = table if table is not None else self.table
+        for p in self.projs:
+            cwl.cwl_apply(self.X[p.d_in], p.W, None if dense else p.A, None if dense else p.B, tab,
+                          self.policy.window, Y=p.Y, workspace=self.apply_ws, status_word=self.status)
+
+    def step(self) -> None:
+        """One pass of the whole hot path on the current stream (no host synchronisation)."""
+        if self.logits is not None:
+            self.score_step()
+        if not self.fixed_table:
+            self.partition_step()
+        self.apply_step()
+
+    def launches_per_step(self) -> int:
+        n = self.LAUNCHES_APPLY * len(self.projs)
+        if self.logits is not None:
+            n += self.LAUNCHES_SCORE
+        if not self.fixed_table:
+            n += self.LAUNCHES_PARTITION
+        return n

@@ -55,6 +55,7 @@ def test_argument_errors_are_reported_without_a_device(lib_path):
     L = binding.lib()
     # NULL pointers and bad sizes are rejected before anything touches CUDA
     assert L.cwl_score_tokens(None, 8, 4, 8, None, None) == 1
+    assert L.cwl_score_tokens(None, 8, 0, 8, None, None) == 0             # nothing to do
     pol = binding.make_policy([4, 8], [1.0, 1.0], [0.5], 4, 2, 0)     # max_len < min_len
     tab = binding.CChunkTable(8, 8, 8, 8, 8, 8, 4)
     assert L.cwl_partition(8, 8, 1, 16, ctypes.byref(pol), tab, 8, 1 << 20, None, None) == 1
