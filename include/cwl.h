@@ -125,6 +125,29 @@ cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64_t ldw,
                      void* workspace, size_t workspace_bytes,
                      int32_t* status_word, void* stream);
 
+/* No counterpart in the paper: a variant of cwl_apply for callers that cannot allocate device
+ * memory -- code running inside another framework's memory pool, inside a region where cudaMalloc
+ * is forbidden, or on a budget that was fixed before this library was loaded.  It takes no
+ * workspace: the shrink partials and the gated H' live in an array of CWL_NOALLOC_SCRATCH_BYTES
+ * bytes that is part of the library image (each GPU that loads the library holds it until the
+ * process exits).  Inputs and outputs are still the caller's.  Same arithmetic, arguments, shape
+ * rules and errors as cwl_apply, plus:
+ *   - CWL_ERR_WORKSPACE when cwl_apply_workspace_bytes(T, d_in, d_out, R) exceeds
+ *     CWL_NOALLOC_SCRATCH_BYTES (with R = 64 every T up to 8192 rows fits); nothing runs.
+ *   - The first call on each device looks the array's device address up (once, with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls share the one array and it keeps whatever the previous call left in it.  Nothing in
+ *     it has to start at zero (every entry that is read was written earlier in the same call), but two
+ *     calls whose kernels overlap on the GPU -- different streams, or the same stream on two host
+ *     threads -- race on it.  Serialise them.
+ * The call allocates nothing on the device and calls no allocating CUDA or framework routine. */
+#define CWL_NOALLOC_SCRATCH_BYTES (8u << 20)
+cwl_status cwl_apply_noalloc(const void* X, int64_t ldx, const void* W, int64_t ldw,
+                             const void* A, int64_t lda, const void* B, int64_t ldb,
+                             int32_t T, int32_t d_in, int32_t d_out, int32_t R,
+                             cwl_chunk_table table, int32_t window,
+                             void* Y, int64_t ldy, int32_t* status_word, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -20,7 +20,8 @@ STATUS = {0: "CWL_OK", 1: "CWL_ERR_INVALID_ARG", 2: "CWL_ERR_SHAPE", 3: "CWL_ERR
           4: "CWL_ERR_CAPACITY", 5: "CWL_ERR_WORKSPACE", 6: "CWL_ERR_CUDA", 7: "CWL_ERR_TIMEOUT"}
 
 EXPORTS = ["cwl_status_string", "cwl_version", "cwl_score_tokens", "cwl_partition_workspace_bytes",
-           "cwl_partition", "cwl_apply_workspace_bytes", "cwl_apply"]
+           "cwl_partition", "cwl_apply_workspace_bytes", "cwl_apply", "cwl_apply_noalloc"]
+NOALLOC_SCRATCH_BYTES = 8 << 20
 
 
 class CwlError(RuntimeError):
@@ -72,6 +73,10 @@ def lib():
                                 C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                 CChunkTable, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t,
                                 C.c_void_p, C.c_void_p]
+        L.cwl_apply_noalloc.restype = C.c_int
+        L.cwl_apply_noalloc.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
+                                        C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                        CChunkTable, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -203,6 +208,23 @@ def cwl_apply(X: torch.Tensor, W: torch.Tensor, A: Optional[torch.Tensor], B: Op
                                         _p(A), A.stride(0) if R else 0, _p(B), B.stride(0) if R else 0,
                                         T, d_in, d_out, R, ct, int(window), _p(Y), Y.stride(0),
                                         _p(workspace), workspace.numel(), _p(status_word), _stream_ptr(stream)))
+    return Y
+
+
+def cwl_apply_noalloc(X: torch.Tensor, W: torch.Tensor, A: Optional[torch.Tensor], B: Optional[torch.Tensor],
+                      table: Optional[DeviceChunkTable], window: int, Y: torch.Tensor,
+                      status_word: Optional[torch.Tensor] = None,
+                      stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """cwl_apply for callers that cannot allocate on the device: no workspace argument, the scratch
+    is the library's own fixed array (NOALLOC_SCRATCH_BYTES).  ``Y`` must be supplied by the caller;
+    this wrapper creates no tensor.  Calls that overlap on the GPU race on the shared scratch."""
+    T, d_in = X.shape
+    d_out = W.shape[1]
+    R = A.shape[1] if (A is not None and B is not None) else 0
+    ct = table.c_struct() if table is not None else CChunkTable(None, None, None, None, None, None, 0)
+    _check("cwl_apply_noalloc", lib().cwl_apply_noalloc(
+        _p(X), X.stride(0), _p(W), W.stride(0), _p(A), A.stride(0) if R else 0, _p(B), B.stride(0) if R else 0,
+        T, d_in, d_out, R, ct, int(window), _p(Y), Y.stride(0), _p(status_word), _stream_ptr(stream)))
     return Y
 
 

@@ -619,3 +619,50 @@ extern "C" cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64
   if (adapter) return launch_gemm<256, 4, MODE_PROJECT>(mX, mW, mH, mB, gp, stream);
   return launch_gemm<256, 4, MODE_PROJECT>(mX, mW, mX, mW, gp, stream);
 }
+
+// ------------------------------------------------------------------------------ no-allocation variant
+// Scratch for cwl_apply_noalloc lives in the library image itself, so a caller that may not allocate
+// device memory (no cudaMalloc in its context, or an allocator it does not own) can still run the
+// adapted projection.  Every device that loads the library carries this array until the process exits.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[CWL_NOALLOC_SCRATCH_BYTES];
+
+namespace cwl {
+namespace {
+
+// Device address of g_noalloc_scratch on the current device.  The array's name is only a host-side
+// handle here; the address the kernels need comes from cudaGetSymbolAddress, once per device.
+cwl_status noalloc_scratch(void** out) {
+  static std::mutex mu;
+  static void* ptr_of_device[64] = {};
+  int dev = 0;
+  CWL_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return CWL_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(mu);
+  if (ptr_of_device[dev] == nullptr) {
+    void* p = nullptr;
+    CWL_CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+    if (p == nullptr) return CWL_ERR_CUDA;
+    ptr_of_device[dev] = p;
+  }
+  *out = ptr_of_device[dev];
+  return CWL_OK;
+}
+
+}  // namespace
+}  // namespace cwl
+
+extern "C" cwl_status cwl_apply_noalloc(const void* X, int64_t ldx, const void* W, int64_t ldw,
+                                        const void* A, int64_t lda, const void* B, int64_t ldb,
+                                        int32_t T, int32_t d_in, int32_t d_out, int32_t R,
+                                        cwl_chunk_table table, int32_t window,
+                                        void* Y, int64_t ldy, int32_t* status_word, void* stream) {
+  if (T < 0 || d_in < 1 || d_out < 1 || R < 0) return CWL_ERR_INVALID_ARG;
+  const bool adapter = (A != nullptr && B != nullptr && R > 0);
+  if (adapter && T > 0 && cwl_apply_workspace_bytes(T, d_in, d_out, R) > (size_t)CWL_NOALLOC_SCRATCH_BYTES)
+    return CWL_ERR_WORKSPACE;  // the problem needs more scratch than the built-in array holds
+  void* scratch = nullptr;
+  const cwl_status st = cwl::noalloc_scratch(&scratch);
+  if (st != CWL_OK) return st;
+  return cwl_apply(X, ldx, W, ldw, A, lda, B, ldb, T, d_in, d_out, R, table, window, Y, ldy, scratch,
+                   (size_t)CWL_NOALLOC_SCRATCH_BYTES, status_word, stream);
+}
