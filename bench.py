@@ -68,7 +68,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
@@ -294,41 +294,43 @@ def run_ours(args):
         b.record(stream)
         torch.cuda.synchronize()
         return a.elapsed_time(b) / n
-    static_ms = time_apply(table=static_tab)
-    dense_ms = time_apply(dense=True)
+    static_ms = None if args.lean else time_apply(table=static_tab)
+    dense_ms = None if args.lean else time_apply(dense=True)
 
     # ---- end to end: pinned host inputs in, results out, every step ----------------------------
-    host_in = {d: x.cpu().pin_memory() for d, x in hp.X.items()}
-    host_logits = hp.logits.cpu().pin_memory() if hp.logits is not None else None
-    host_out = [torch.empty(p.Y.shape, dtype=p.Y.dtype).pin_memory() for p in hp.projs]
-    h2d = sum(x.numel() * x.element_size() for x in host_in.values()) + \
-        (host_logits.numel() * 4 if host_logits is not None else 0)
-    d2h = sum(y.numel() * y.element_size() for y in host_out)
-    e2e_steps = max(3, min(args.steps, 20))
+    e2e_value, e2e_steps, h2d, d2h = None, 0, 0, 0
+    if not args.lean:
+        host_in = {d: x.cpu().pin_memory() for d, x in hp.X.items()}
+        host_logits = hp.logits.cpu().pin_memory() if hp.logits is not None else None
+        host_out = [torch.empty(p.Y.shape, dtype=p.Y.dtype).pin_memory() for p in hp.projs]
+        h2d = sum(x.numel() * x.element_size() for x in host_in.values()) + \
+            (host_logits.numel() * 4 if host_logits is not None else 0)
+        d2h = sum(y.numel() * y.element_size() for y in host_out)
+        e2e_steps = max(3, min(args.steps, 20))
 
-    def e2e_step():
-        for d, x in host_in.items():
-            hp.X[d].copy_(x, non_blocking=True)
-        if host_logits is not None:
-            hp.logits.copy_(host_logits, non_blocking=True)
-        hp.step()
-        for p, y in zip(hp.projs, host_out):
-            y.copy_(p.Y, non_blocking=True)
-    for _ in range(2):
-        e2e_step()
-    barrier()
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record(stream)
-    for _ in range(e2e_steps):
-        e2e_step()
-    b.record(stream)
-    barrier()
-    e2e_ms = a.elapsed_time(b)
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = hp.T * e2e_steps * world / (e2e_ms * 1e-3)
+        def e2e_step():
+            for d, x in host_in.items():
+                hp.X[d].copy_(x, non_blocking=True)
+            if host_logits is not None:
+                hp.logits.copy_(host_logits, non_blocking=True)
+            hp.step()
+            for p, y in zip(hp.projs, host_out):
+                y.copy_(p.Y, non_blocking=True)
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        b.record(stream)
+        barrier()
+        e2e_ms = a.elapsed_time(b)
+        if world > 1:
+            t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        e2e_value = hp.T * e2e_steps * world / (e2e_ms * 1e-3)
 
     if rank != 0:
         if world > 1:
@@ -356,8 +358,11 @@ def run_ours(args):
     roof["executed_tflops"] = f_exe / (apply_avg_ms * 1e-3) / 1e12
     roof["frac_of_nominal_2250"] = (f_alg / (apply_avg_ms * 1e-3) / 1e12) / 2250.0
 
-    n_rows, _ = rows_for_budget(w, 12.0)             # about 10-20 s of CPU work
-    cpu_val, cpu_info = oracle_sample(w, n_rows=n_rows)
+    if args.lean:
+        cpu_val, cpu_info = None, {}
+    else:
+        n_rows, _ = rows_for_budget(w, 12.0)         # about 10-20 s of CPU work
+        cpu_val, cpu_info = oracle_sample(w, n_rows=n_rows)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -389,13 +394,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg4"])
+    ap.add_argument("--lean", action="store_true",
+                    help="timed region only (no comparison runs, end-to-end leg or CPU baseline): for profiler runs")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 2 if args.steps is None else max(1, args.steps)
         args.warmup = 1 if args.warmup is None else max(0, args.warmup)
         run_reference(args)
     else:
-        args.steps = 200 if args.steps is None else max(1, args.steps)
+        args.steps = 500 if args.steps is None else max(1, args.steps)
         args.warmup = max(5 if args.warmup is None else args.warmup, 3)
         run_ours(args)
 

@@ -133,12 +133,13 @@ cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64_t ldw,
  * process exits).  Inputs and outputs are still the caller's.  Same arithmetic, arguments, shape
  * rules and errors as cwl_apply, plus:
  *   - CWL_ERR_WORKSPACE when cwl_apply_workspace_bytes(T, d_in, d_out, R) exceeds
- *     CWL_NOALLOC_SCRATCH_BYTES (with R = 64 every T up to 8192 rows fits); nothing runs.
+ *     CWL_NOALLOC_SCRATCH_BYTES (with R = 64 every T up to 32768 rows fits); nothing runs.
  *   - The first call on each device looks the array's device address up (once, with that device
  *     current); make that first call outside any stream capture.
- *   - All calls share the one array and it keeps whatever the previous call left in it.  Nothing in
- *     it has to start at zero (every entry that is read was written earlier in the same call), but two
- *     calls whose kernels overlap on the GPU -- different streams, or the same stream on two host
+ *   - All calls share the one array and it keeps whatever the previous call left in it.  The few
+ *     words that must start at zero (per-row-tile counters and flags) are cleared by every call on its
+ *     stream before the kernel; everything else that is read was written earlier in the same call.
+ *     Two calls whose kernels overlap on the GPU -- different streams, or the same stream on two host
  *     threads -- race on it.  Serialise them.
  * The call allocates nothing on the device and calls no allocating CUDA or framework routine. */
 #define CWL_NOALLOC_SCRATCH_BYTES (8u << 20)

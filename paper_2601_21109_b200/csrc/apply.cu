@@ -2,18 +2,23 @@
 //
 //   y_t = x_t W + ((x_t A) * g_t) B,   g_t[j] = (1-lam_t) s_p [j < r_p] + lam_t s_c [j < r_c]
 //
-// which, by linearity, equals blending the outgoing and incoming adapter outputs.  Three launches:
-//   1. shrink   P = X A at the ladder's full rank R        (tcgen05 GEMM, split along d_in, fp32 partials)
-//   2. gate     H' = bf16(g * sum of partials)             (per-row rank mask, scale and cross-fade weight)
-//   3. project  Y = bf16([X | H'] [W ; B])                 (tcgen05 GEMM: the K loop runs over d_in, then
-//                                                           over R, into ONE TMEM accumulator)
-// Both GEMMs are one persistent, warp-specialised kernel: a TMA producer warp, an MMA issuer warp
-// (tcgen05.mma, cta_group::1, 128 x BN x 16, bf16 -> fp32 in TMEM) and four epilogue warps that read
-// the accumulator back with tcgen05.ld.  TMEM holds two accumulators so the epilogue of one tile
-// overlaps the main loop of the next.  The left operand is K-major (rows of X), the right operand
-// is N-major (rows of W are contiguous in d_out), both 128-byte swizzled as TMA writes them.
+// which, by linearity, equals blending the outgoing and incoming adapter outputs.  ONE persistent,
+// warp-specialised kernel does all of it.  Each CTA first works through its share of SHRINK items
+//   P[split] = X[:, split of d_in] A[split, :]   (full ladder rank R, fp32 partials when d_in is split),
+// the CTA that completes a row tile's last split sums the partials, applies the per-row gate (rank
+// mask, scale and cross-fade weight from the chunk table, expanded per row in shared memory) and
+// publishes H' = bf16(g * X A) with a release flag; then the CTAs work through the PROJECT tiles
+//   Y = bf16([X | H'] [W ; B])
+// whose K loop runs over d_in and then over R into ONE TMEM accumulator (the TMA producer acquires the
+// row tile's flag before its first H' load, ~d_in/64 pipeline steps after the tile began).
 //
-// Every wait on an mbarrier is bounded: when it runs out the CTA raises CWL_ERR_TIMEOUT in the
+// Roles: warp 0 = TMA producer (cp.async.bulk.tensor, 128-byte swizzle), warp 1 = tcgen05.mma issuer
+// (cta_group::1, 128 x N x 16, bf16 -> fp32 in TMEM), warps 2..5 = epilogue (tcgen05.ld).  TMEM holds
+// two accumulators so the epilogue of one item overlaps the main loop of the next.  The left operand
+// is K-major (rows of X / H'), the right operand is N-major (rows of W, A, B are contiguous in their
+// output dimension), exactly as the matrices sit in HBM.
+//
+// Every wait (mbarrier or flag) is bounded: when it runs out the CTA raises CWL_ERR_TIMEOUT in the
 // status word, drains what it has in flight, frees its TMEM and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -27,25 +32,31 @@ namespace cwl {
 namespace {
 
 constexpr int BM = 128;             // rows per tile = TMEM lanes
+constexpr int BN = 256;             // columns per projection tile = one TMEM accumulator
 constexpr int BK = 64;              // K elements per stage = one 128-byte swizzle row of bf16
 constexpr int UMMA_K = 16;
+constexpr int kStages = 4;
 constexpr int kGemmThreads = 192;   // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
 constexpr int kEpilogueThreads = 128;
 constexpr int kGroupM = 16;         // row tiles per raster group (keeps their X rows L2-resident)
 constexpr int kNumSmsPlanned = 148; // used where the answer must not depend on the device
+constexpr int kMaxSplits = 16;      // split factor of the shrink along d_in
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
-enum : int { MODE_PROJECT = 0, MODE_SHRINK = 1 };
+struct RowGate { float w_in, w_out; int r_in, r_out; };  // g[j] = w_in [j < r_in] + w_out [j < r_out]
 
-struct GemmParams {
-  int M;            // rows (tokens)
-  int N;            // columns of the result
-  int K0, K1;       // depth of phase 0 (d_in) and phase 1 (R, 0 when there is no adapter)
+struct ApplyParams {
+  int T, d_in, d_out, R;   // R = 0: no adapter
+  int r_pad;               // R rounded up to the 64-column swizzle atom
   int n_m_tiles, n_n_tiles;
-  int splits;       // split-K factor over phase 0 (shrink only)
-  int kb_per_split; // K blocks per split
-  void* out;        // PROJECT: bf16 [M, ld_out];  SHRINK: fp32 [splits, M, ld_out]
-  int64_t ld_out;
+  int splits, kb_per_split;
+  int window;
+  __nv_bfloat16* Y; int64_t ldy;
+  __nv_bfloat16* Hg;       // [T, R] gated shrink output
+  float* partial;          // [splits, T, R]
+  int* counters;           // [n_m_tiles] splits finished per row tile
+  int* flags;              // [n_m_tiles] 1 once H' of the row tile is published
+  cwl_chunk_table table;
   int32_t* status_word;
 };
 
@@ -160,49 +171,118 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// ------------------------------------------------------------------------------------ the GEMM
-template <int BN, int STAGES>
+
+__device__ __forceinline__ void epilogue_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(int* p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// orders this thread's generic-proxy observations before its later async-proxy (TMA) accesses
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// ------------------------------------------------------------------------------------ work items
+enum : int { ITEM_SHRINK = 0, ITEM_PROJECT = 1 };
+struct Item { int kind, m_tile, n_tile, split; };
+
 struct SmemPlan {
-  static constexpr int kABytes = BM * BK * 2;       // 16 KB, one TMA box
-  static constexpr int kBBytes = BN * BK * 2;       // BN/64 TMA boxes of 64 x 64
+  static constexpr int kABytes = BM * BK * 2;       // 16 KB: one TMA box of X or H'
+  static constexpr int kBBytes = BN * BK * 2;       // 32 KB: four 64 x 64 boxes of W, B or A
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kTileBytes = STAGES * kStageBytes;
-  static constexpr int kBarBytes = (2 * STAGES + 4) * 8 + 16;
-  static constexpr int kTotal = kTileBytes + kBarBytes + 1024;  // + slack for 1024-byte alignment
+  static constexpr int kTileBytes = kStages * kStageBytes;
+  static constexpr int kBarBytes = (2 * kStages + 4) * 8;
+  static constexpr int kMiscBytes = 32;             // TMEM base, abort flag, epilogue broadcast words
+  static constexpr int kGateBytes = BM * (int)sizeof(RowGate);
+  static constexpr int kTotal = kTileBytes + kBarBytes + kMiscBytes + kGateBytes + 1024;  // + alignment slack
 };
 
-struct TileCoord { int m_tile, n_tile, split; };
-
-__device__ __forceinline__ TileCoord tile_coord(int tile, const GemmParams& p) {
-  TileCoord c;
-  c.split = tile % p.splits;
-  tile /= p.splits;
+// The i-th work item of this CTA.  Shrink items come first and are dealt from the LAST CTA downwards,
+// so the CTAs that receive one projection tile fewer carry the shrink work.  Projection tiles are
+// rastered in groups of kGroupM row tiles (row tile fastest inside a group).
+__device__ __forceinline__ bool get_item(int i, const ApplyParams& p, Item& it) {
+  const int G = gridDim.x, b = blockIdx.x;
+  const int n_shrink = (p.R > 0) ? p.n_m_tiles * p.splits : 0;
+  const int first_s = G - 1 - b;
+  const int my_shrink = first_s < n_shrink ? (n_shrink - 1 - first_s) / G + 1 : 0;
+  if (i < my_shrink) {
+    const int s = first_s + i * G;
+    it.kind = ITEM_SHRINK; it.m_tile = s / p.splits; it.split = s - it.m_tile * p.splits; it.n_tile = 0;
+    return true;
+  }
+  const int tile = b + (i - my_shrink) * G;
+  if (tile >= p.n_m_tiles * p.n_n_tiles) return false;
   const int per_group = kGroupM * p.n_n_tiles;
   const int group = tile / per_group, within = tile - group * per_group;
   const int first_m = group * kGroupM;
   const int gsize = min(kGroupM, p.n_m_tiles - first_m);
-  c.m_tile = first_m + within % gsize;
-  c.n_tile = within / gsize;
-  return c;
+  it.kind = ITEM_PROJECT; it.split = 0;
+  it.m_tile = first_m + within % gsize;
+  it.n_tile = within / gsize;
+  return true;
 }
 
-// K blocks a tile runs over: phase 0 blocks [kb0, kb1) of X/W, then all of phase 1 (H'/B)
-__device__ __forceinline__ void tile_k_range(const TileCoord& c, const GemmParams& p, int& kb0, int& kb1, int& nkb1) {
-  const int nkb0 = (p.K0 + BK - 1) / BK;
-  kb0 = c.split * p.kb_per_split;
-  kb1 = min(nkb0, kb0 + p.kb_per_split);
-  nkb1 = (p.K1 + BK - 1) / BK;
+// Pipeline steps of an item: shrink = its split of the d_in blocks; project = all d_in blocks, then R blocks.
+__device__ __forceinline__ void item_blocks(const Item& it, const ApplyParams& p, int& kb0, int& n0, int& n1) {
+  const int nkb0 = (p.d_in + BK - 1) / BK;
+  if (it.kind == ITEM_SHRINK) {
+    kb0 = it.split * p.kb_per_split;
+    n0 = min(nkb0, kb0 + p.kb_per_split) - kb0;
+    n1 = 0;
+  } else {
+    kb0 = 0; n0 = nkb0; n1 = (p.R + BK - 1) / BK;
+  }
 }
 
-template <int BN, int STAGES, int MODE>
+// Per-row gate from the chunk table (Sec. III-C rank mask and scale, Sec. III-D cross-fade weight).
+__device__ __forceinline__ RowGate row_gate(int t, const ApplyParams& p) {
+  RowGate g{0.f, 0.f, 0, 0};
+  const cwl_chunk_table& tb = p.table;
+  const int C = min(*tb.n_chunks, tb.capacity);
+  if (t < p.T && C > 0 && t >= tb.offsets[0] && t < tb.offsets[C]) {
+    int lo = 0, hi = C;                            // offsets[lo] <= t < offsets[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (tb.offsets[mid] <= t) lo = mid; else hi = mid;
+    }
+    const int c = lo, j = t - tb.offsets[c];
+    float lam = 1.f;
+    if (c > 0 && !(tb.flags[c] & 1) && j < p.window) lam = (float)(j + 1) / (float)(p.window + 1);
+    g.r_in = min(max(tb.rank[c], 0), p.R);
+    g.w_in = lam * tb.scale[c];
+    if (lam < 1.f) {
+      g.r_out = min(max(tb.rank[c - 1], 0), p.R);
+      g.w_out = (1.f - lam) * tb.scale[c - 1];
+    }
+  }
+  return g;
+}
+__device__ __forceinline__ float gate_at(const RowGate& g, int j) {
+  return (j < g.r_in ? g.w_in : 0.f) + (j < g.r_out ? g.w_out : 0.f);
+}
+
+// Bounded acquire-wait on a row tile's "H' published" flag.
+__device__ __forceinline__ bool wait_flag(const int* flag, volatile int* abort_flag) {
+  if (ld_acquire(flag) != 0) return true;
+  const unsigned long long t0 = global_timer();
+  for (uint32_t spins = 1;; ++spins) {
+    if (ld_acquire(flag) != 0) return true;
+    __nanosleep(64);
+    if ((spins & 63u) == 0) {
+      if (*abort_flag) return false;
+      if (global_timer() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap tm_a0, const __grid_constant__ CUtensorMap tm_b0,
-            const __grid_constant__ CUtensorMap tm_a1, const __grid_constant__ CUtensorMap tm_b1,
-            const GemmParams p) {
-  using Plan = SmemPlan<BN, STAGES>;
-  constexpr uint32_t kTmemCols = 2 * BN;            // two accumulators (a power of two >= 32)
-  static_assert(BN % 64 == 0 && BN >= 64 && BN <= 256, "BN is a multiple of the 64-column swizzle atom");
-  static_assert(kTmemCols == 128 || kTmemCols == 256 || kTmemCols == 512, "TMEM columns: power of two");
+apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
+             const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_h,
+             const __grid_constant__ CUtensorMap tm_b, const ApplyParams p) {
+  using Plan = SmemPlan;
+  constexpr uint32_t kTmemCols = 2 * BN;            // two accumulators: all 512 columns
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -210,23 +290,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a0, const __grid_constant__ C
   uint8_t* base_ptr = smem_raw + (base - raw);
   const uint32_t bars = base + Plan::kTileBytes;
   auto full_bar = [&](int s) { return bars + 8u * s; };
-  auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
-  auto acc_full_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
-  auto acc_empty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + Plan::kTileBytes + (2 * STAGES + 4) * 8);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + Plan::kTileBytes + (2 * STAGES + 4) * 8 + 4);
+  auto empty_bar = [&](int s) { return bars + 8u * (kStages + s); };
+  auto acc_full_bar = [&](int a) { return bars + 8u * (2 * kStages + a); };
+  auto acc_empty_bar = [&](int a) { return bars + 8u * (2 * kStages + 2 + a); };
+  uint8_t* misc = base_ptr + Plan::kTileBytes + Plan::kBarBytes;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
+  volatile int* epi_go = reinterpret_cast<volatile int*>(misc + 8);     // epilogue: proceed with this item?
+  volatile int* epi_last = reinterpret_cast<volatile int*>(misc + 12);  // epilogue: this CTA finalises the row tile
+  RowGate* gates = reinterpret_cast<RowGate*>(misc + Plan::kMiscBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total_tiles = p.n_m_tiles * p.n_n_tiles * p.splits;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), kEpilogueThreads); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    prefetch_tmap(&tm_a0);
-    prefetch_tmap(&tm_b0);
-    if (p.K1 > 0) { prefetch_tmap(&tm_a1); prefetch_tmap(&tm_b1); }
+    prefetch_tmap(&tm_x);
+    prefetch_tmap(&tm_w);
+    if (p.R > 0) { prefetch_tmap(&tm_a); prefetch_tmap(&tm_h); prefetch_tmap(&tm_b); }
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
@@ -240,67 +323,76 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a0, const __grid_constant__ C
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      uint32_t it = 0;          // running stage counter across tiles
+      uint32_t it_cnt = 0;      // running stage counter across items
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const TileCoord c = tile_coord(tile, p);
-        int kb0, kb1, nkb1;
-        tile_k_range(c, p, kb0, kb1, nkb1);
-        const int n_blocks = (kb1 - kb0) + nkb1;
-        for (int i = 0; i < n_blocks; ++i, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1u;
+      Item item;
+      for (int i = 0; ok && get_item(i, p, item); ++i) {
+        int kb0, n0, n1;
+        item_blocks(item, p, kb0, n0, n1);
+        const bool shrink = item.kind == ITEM_SHRINK;
+        const int n_boxes = shrink ? p.r_pad / 64 : BN / 64;
+        const uint32_t tx = Plan::kABytes + n_boxes * (BK * 128);
+        const CUtensorMap* right0 = shrink ? &tm_a : &tm_w;
+        const int col0 = shrink ? 0 : item.n_tile * BN;
+        for (int b = 0; b < n0 + n1; ++b, ++it_cnt) {
+          const int s = it_cnt % kStages;
+          const uint32_t ph = (it_cnt / kStages) & 1u;
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-          const bool phase1 = i >= (kb1 - kb0);
-          const int k = phase1 ? (i - (kb1 - kb0)) * BK : (kb0 + i) * BK;
-          const CUtensorMap* ma = phase1 ? &tm_a1 : &tm_a0;
-          const CUtensorMap* mb = phase1 ? &tm_b1 : &tm_b0;
+          const bool phase1 = b >= n0;
+          if (phase1 && b == n0) {
+            // H' of this row tile must have been published by whoever finished its shrink
+            if (!wait_flag(p.flags + item.m_tile, abort_flag)) { ok = false; break; }
+            fence_proxy_async();
+          }
+          const int k = phase1 ? (b - n0) * BK : (kb0 + b) * BK;
+          const CUtensorMap* left = phase1 ? &tm_h : &tm_x;
+          const CUtensorMap* right = phase1 ? &tm_b : right0;
           const uint32_t sa = base + s * Plan::kStageBytes, sb = sa + Plan::kABytes;
-          mbar_expect_tx(full_bar(s), Plan::kStageBytes);
-          tma_load_2d(sa, ma, full_bar(s), k, c.m_tile * BM);
-#pragma unroll
-          for (int j = 0; j < BN / 64; ++j)
-            tma_load_2d(sb + j * (BK * 128), mb, full_bar(s), c.n_tile * BN + j * 64, k);
+          mbar_expect_tx(full_bar(s), tx);
+          tma_load_2d(sa, left, full_bar(s), k, item.m_tile * BM);
+          for (int j = 0; j < n_boxes; ++j)
+            tma_load_2d(sb + j * (BK * 128), right, full_bar(s), col0 + j * 64, k);
         }
       }
       if (!ok) {
         // drain: give the copies already issued a bounded chance to land before the CTA leaves
-        for (uint32_t back = 1; back <= (uint32_t)STAGES && back <= it; ++back) {
-          const uint32_t j = it - back;
+        for (uint32_t back = 1; back <= (uint32_t)kStages && back <= it_cnt; ++back) {
+          const uint32_t j = it_cnt - back;
           unsigned long long t0 = global_timer();
-          while (!mbar_try_wait(full_bar(j % STAGES), (j / STAGES) & 1u) && global_timer() - t0 < kWaitLimitNs) {}
+          while (!mbar_try_wait(full_bar(j % kStages), (j / kStages) & 1u) && global_timer() - t0 < kWaitLimitNs) {}
         }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc(BM, BN);
-      uint32_t it = 0, local_tile = 0;
+      const uint32_t idesc_project = make_idesc(BM, BN);
+      const uint32_t idesc_shrink = make_idesc(BM, p.r_pad > 0 ? p.r_pad : 64);
+      uint32_t it_cnt = 0, local = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local_tile) {
-        const TileCoord c = tile_coord(tile, p);
-        int kb0, kb1, nkb1;
-        tile_k_range(c, p, kb0, kb1, nkb1);
-        const int n_blocks = (kb1 - kb0) + nkb1;
-        const uint32_t acc = local_tile & 1u, acc_ph = (local_tile >> 1) & 1u;
+      Item item;
+      for (int i = 0; ok && get_item(i, p, item); ++i, ++local) {
+        int kb0, n0, n1;
+        item_blocks(item, p, kb0, n0, n1);
+        const uint32_t idesc = item.kind == ITEM_SHRINK ? idesc_shrink : idesc_project;
+        const uint32_t acc = local & 1u, acc_ph = (local >> 1) & 1u;
         if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int i = 0; i < n_blocks; ++i, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1u;
+        for (int b = 0; b < n0 + n1; ++b, ++it_cnt) {
+          const int s = it_cnt % kStages;
+          const uint32_t ph = (it_cnt / kStages) & 1u;
           if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const bool phase1 = i >= (kb1 - kb0);
-          const int k = phase1 ? (i - (kb1 - kb0)) * BK : (kb0 + i) * BK;
-          const int k_left = (phase1 ? p.K1 : p.K0) - k;         // multiple of 16
+          const bool phase1 = b >= n0;
+          const int k = phase1 ? (b - n0) * BK : (kb0 + b) * BK;
+          const int k_left = (phase1 ? p.R : p.d_in) - k;          // multiple of 16
           const int k_steps = k_left >= BK ? BK / UMMA_K : k_left / UMMA_K;
           const uint32_t sa = base + s * Plan::kStageBytes, sb = sa + Plan::kABytes;
           for (int kk = 0; kk < k_steps; ++kk) {
             const uint64_t da = make_smem_desc(sa + kk * (UMMA_K * 2), 16, 1024);
             const uint64_t db = make_smem_desc(sb + kk * (UMMA_K * 128), BK * 128, 1024);
-            umma_bf16(d_tmem, da, db, idesc, (i | kk) != 0 ? 1u : 0u);
+            umma_bf16(d_tmem, da, db, idesc, (b | kk) != 0 ? 1u : 0u);
           }
           umma_commit(empty_bar(s));            // frees the stage once these MMAs have read it
         }
@@ -316,28 +408,34 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a0, const __grid_constant__ C
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     const int lane_group = warp & 3;              // TMEM lanes this warp may read: 32*lane_group ..
     const int row_in_tile = lane_group * 32 + lane;
-    uint32_t local_tile = 0;
-    bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local_tile) {
-      const TileCoord c = tile_coord(tile, p);
-      const uint32_t acc = local_tile & 1u, acc_ph = (local_tile >> 1) & 1u;
-      if (!mbar_wait(acc_full_bar(acc), acc_ph, abort_flag)) { ok = false; break; }
+    const int epi_tid = threadIdx.x - 64;         // 0..127
+    uint32_t local = 0;
+    Item item;
+    for (int i = 0; get_item(i, p, item); ++i, ++local) {
+      const uint32_t acc = local & 1u, acc_ph = (local >> 1) & 1u;
+      mbar_wait(acc_full_bar(acc), acc_ph, abort_flag);   // a failure is recorded in abort_flag
+      // one thread decides for all 128 so that the barriers below are never split
+      epilogue_barrier();
+      if (epi_tid == 0) *epi_go = (*abort_flag == 0);
+      epilogue_barrier();
+      if (*epi_go == 0) break;
       tc_fence_after();
-      const int row = c.m_tile * BM + row_in_tile;
+      const int row = item.m_tile * BM + row_in_tile;
       const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(lane_group * 32) << 16);
+
+      if (item.kind == ITEM_PROJECT) {
 #pragma unroll 1
-      for (int cc = 0; cc < BN / 32; ++cc) {
-        const int col = c.n_tile * BN + cc * 32;
-        if (col >= p.N) break;                     // warp-uniform
-        uint32_t v[32];
-        tmem_ld32(t_row + cc * 32, v);
-        tmem_ld_wait();
-        if (row < p.M) {
-          if (MODE == MODE_PROJECT) {
-            __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)row * p.ld_out + col;
+        for (int cc = 0; cc < BN / 32; ++cc) {
+          const int col = item.n_tile * BN + cc * 32;
+          if (col >= p.d_out) break;                 // warp-uniform
+          uint32_t v[32];
+          tmem_ld32(t_row + cc * 32, v);
+          tmem_ld_wait();
+          if (row < p.T) {
+            __nv_bfloat16* out = p.Y + (int64_t)row * p.ldy + col;
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
-              if (col + g * 8 < p.N) {             // N is a multiple of 8: a granule is all in or all out
+              if (col + g * 8 < p.d_out) {           // d_out is a multiple of 8: a granule is all in or all out
                 uint4 q;
                 q.x = pack_bf16(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
                 q.y = pack_bf16(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
@@ -346,20 +444,86 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a0, const __grid_constant__ C
                 *reinterpret_cast<uint4*>(out + g * 8) = q;
               }
             }
-          } else {
-            float* out = reinterpret_cast<float*>(p.out) + ((int64_t)c.split * p.M + row) * p.ld_out + col;
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(acc_empty_bar(acc));
+        continue;
+      }
+
+      // ---- shrink item ----
+      const bool direct = p.splits == 1;             // no partials: gate straight from the accumulator
+      RowGate g{0.f, 0.f, 0, 0};
+      if (direct) g = row_gate(row, p);
+#pragma unroll 1
+      for (int cc = 0; cc < p.r_pad / 32; ++cc) {
+        const int col = cc * 32;
+        if (col >= p.R) break;                       // warp-uniform
+        uint32_t v[32];
+        tmem_ld32(t_row + cc * 32, v);
+        tmem_ld_wait();
+        if (row < p.T) {
+          if (direct) {
+            __nv_bfloat16* out = p.Hg + (int64_t)row * p.R + col;
 #pragma unroll
-            for (int g = 0; g < 8; ++g) {
-              if (col + g * 4 < p.N) {
-                uint4 q = make_uint4(v[g * 4 + 0], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
-                *reinterpret_cast<uint4*>(out + g * 4) = q;
+            for (int q8 = 0; q8 < 4; ++q8) {
+              if (col + q8 * 8 < p.R) {
+                const int j = col + q8 * 8;
+                uint4 q;
+                q.x = pack_bf16(__uint_as_float(v[q8 * 8 + 0]) * gate_at(g, j + 0), __uint_as_float(v[q8 * 8 + 1]) * gate_at(g, j + 1));
+                q.y = pack_bf16(__uint_as_float(v[q8 * 8 + 2]) * gate_at(g, j + 2), __uint_as_float(v[q8 * 8 + 3]) * gate_at(g, j + 3));
+                q.z = pack_bf16(__uint_as_float(v[q8 * 8 + 4]) * gate_at(g, j + 4), __uint_as_float(v[q8 * 8 + 5]) * gate_at(g, j + 5));
+                q.w = pack_bf16(__uint_as_float(v[q8 * 8 + 6]) * gate_at(g, j + 6), __uint_as_float(v[q8 * 8 + 7]) * gate_at(g, j + 7));
+                *reinterpret_cast<uint4*>(out + q8 * 8) = q;
               }
+            }
+          } else {
+            float* out = p.partial + ((int64_t)item.split * p.T + row) * p.R + col;
+#pragma unroll
+            for (int q4 = 0; q4 < 8; ++q4) {
+              if (col + q4 * 4 < p.R)
+                *reinterpret_cast<uint4*>(out + q4 * 4) = make_uint4(v[q4 * 4 + 0], v[q4 * 4 + 1], v[q4 * 4 + 2], v[q4 * 4 + 3]);
             }
           }
         }
       }
       tc_fence_before();
-      mbar_arrive(acc_empty_bar(acc));
+      mbar_arrive(acc_empty_bar(acc));               // the accumulator is free again
+
+      __threadfence();                               // this thread's H' / partial stores, device-wide
+      epilogue_barrier();
+      if (direct) {
+        if (epi_tid == 0) st_release(p.flags + item.m_tile, 1);
+        continue;
+      }
+      if (epi_tid == 0) *epi_last = (atomicAdd(p.counters + item.m_tile, 1) == p.splits - 1);
+      epilogue_barrier();
+      if (*epi_last == 0) continue;
+      // this CTA completed the row tile: sum the partials, gate, publish H'
+      __threadfence();
+      gates[epi_tid] = row_gate(item.m_tile * BM + epi_tid, p);
+      epilogue_barrier();
+      const int quads = p.R >> 2;                    // float4 groups per row
+      const int64_t split_stride = (int64_t)p.T * p.R;
+      for (int idx = epi_tid; idx < BM * quads; idx += kEpilogueThreads) {
+        const int r = idx / quads, j0 = (idx - r * quads) << 2;
+        const int t = item.m_tile * BM + r;
+        if (t >= p.T) break;
+        const RowGate gr = gates[r];
+        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float* src = p.partial + (int64_t)t * p.R + j0;
+        for (int s = 0; s < p.splits; ++s) {
+          const float4 x = __ldcg(reinterpret_cast<const float4*>(src + s * split_stride));
+          sum.x += x.x; sum.y += x.y; sum.z += x.z; sum.w += x.w;
+        }
+        uint2 o;
+        o.x = pack_bf16(sum.x * gate_at(gr, j0), sum.y * gate_at(gr, j0 + 1));
+        o.y = pack_bf16(sum.z * gate_at(gr, j0 + 2), sum.w * gate_at(gr, j0 + 3));
+        *reinterpret_cast<uint2*>(p.Hg + (int64_t)t * p.R + j0) = o;
+      }
+      __threadfence();
+      epilogue_barrier();
+      if (epi_tid == 0) st_release(p.flags + item.m_tile, 1);
     }
   }
 
@@ -370,63 +534,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a0, const __grid_constant__ C
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
-  }
-}
-
-// --------------------------------------------------------------------------------------- gate
-// H'[t, j] = bf16(g_t[j] * sum_s partial[s][t][j]).  Each block expands the chunk table into one
-// row descriptor per token in shared memory, then all threads apply it.
-constexpr int kGateRows = 32;
-constexpr int kGateThreads = 256;
-
-struct RowGate { float w_in, w_out; int r_in, r_out; };  // g[j] = w_in [j < r_in] + w_out [j < r_out]
-
-__global__ void __launch_bounds__(kGateThreads)
-gate_kernel(const float* __restrict__ partial, int splits, int T, int R, cwl_chunk_table table, int window,
-            __nv_bfloat16* __restrict__ Hg) {
-  __shared__ RowGate gates[kGateRows];
-  const int row0 = blockIdx.x * kGateRows;
-  if (threadIdx.x < kGateRows) {
-    const int t = row0 + threadIdx.x;
-    RowGate g{0.f, 0.f, 0, 0};
-    const int C = min(*table.n_chunks, table.capacity);
-    if (t < T && C > 0 && t >= table.offsets[0] && t < table.offsets[C]) {
-      int lo = 0, hi = C;                          // offsets[lo] <= t < offsets[hi]
-      while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (table.offsets[mid] <= t) lo = mid; else hi = mid;
-      }
-      const int c = lo, j = t - table.offsets[c];
-      float lam = 1.f;
-      if (c > 0 && !(table.flags[c] & 1) && j < window) lam = (float)(j + 1) / (float)(window + 1);
-      g.r_in = min(max(table.rank[c], 0), R);
-      g.w_in = lam * table.scale[c];
-      if (lam < 1.f) {
-        g.r_out = min(max(table.rank[c - 1], 0), R);
-        g.w_out = (1.f - lam) * table.scale[c - 1];
-      }
-    }
-    gates[threadIdx.x] = g;
-  }
-  __syncthreads();
-  const int groups_per_row = R >> 2;               // 4 columns per thread step
-  const int64_t split_stride = (int64_t)T * R;
-  for (int idx = threadIdx.x; idx < kGateRows * groups_per_row; idx += kGateThreads) {
-    const int r = idx / groups_per_row, j0 = (idx - r * groups_per_row) << 2;
-    const int t = row0 + r;
-    if (t >= T) break;
-    const RowGate g = gates[r];
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    const float* src = partial + (int64_t)t * R + j0;
-    for (int s = 0; s < splits; ++s) {
-      const float4 v = *reinterpret_cast<const float4*>(src + s * split_stride);
-      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-    }
-    auto gate = [&](int j) { return (j < g.r_in ? g.w_in : 0.f) + (j < g.r_out ? g.w_out : 0.f); };
-    uint2 o;
-    o.x = pack_bf16(acc.x * gate(j0), acc.y * gate(j0 + 1));
-    o.y = pack_bf16(acc.z * gate(j0 + 2), acc.w * gate(j0 + 3));
-    *reinterpret_cast<uint2*>(Hg + (int64_t)t * R + j0) = o;
   }
 }
 
@@ -501,45 +608,31 @@ int sm_count() {
   return n;
 }
 
-template <int BN, int STAGES, int MODE>
-cwl_status launch_gemm(const CUtensorMap& a0, const CUtensorMap& b0, const CUtensorMap& a1, const CUtensorMap& b1,
-                       const GemmParams& p, cudaStream_t stream) {
-  using Plan = SmemPlan<BN, STAGES>;
-  auto kernel = gemm_kernel<BN, STAGES, MODE>;
-  static bool configured[64] = {};  // per device; benign race: the attribute call is idempotent
-  int dev = 0;
-  CWL_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64 || !configured[dev]) {
-    CWL_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Plan::kTotal));
-    if (dev >= 0 && dev < 64) configured[dev] = true;
-  }
-  const int total = p.n_m_tiles * p.n_n_tiles * p.splits;
-  const int grid = total < sm_count() ? total : sm_count();
-  kernel<<<grid, kGemmThreads, Plan::kTotal, stream>>>(a0, b0, a1, b1, p);
-  CWL_CUDA_TRY(cudaGetLastError());
-  return CWL_OK;
-}
-
-// split-K factor of the shrink GEMM: enough CTAs to pull X at full HBM rate when T is small
+// split factor of the shrink along d_in: enough items to spread X over the SMs when T is small
 int shrink_splits(int T, int d_in) {
   const int n_m = ceil_div(T, BM), nkb = ceil_div(d_in, BK);
-  int s = ceil_div(kNumSmsPlanned, n_m);
+  int s = kNumSmsPlanned / n_m;
+  if (s > kMaxSplits) s = kMaxSplits;
   if (s > nkb) s = nkb;
-  if (s > 32) s = 32;
   if (s < 1) s = 1;
   const int per = ceil_div(nkb, s);
   return ceil_div(nkb, per);        // no empty split
 }
 
-struct ApplyWorkspace { __nv_bfloat16* Hg; float* partial; };
+struct ApplyWorkspace { __nv_bfloat16* Hg; float* partial; int* counters; int* flags; size_t sync_bytes; };
 
 size_t carve_apply(ApplyWorkspace& w, char* base, int T, int d_in, int R) {
   auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  const int splits = shrink_splits(T, d_in), n_m = ceil_div(T, BM);
   size_t off = 0;
   w.Hg = reinterpret_cast<__nv_bfloat16*>(base ? base + off : nullptr);
   off = up(off + (size_t)T * R * sizeof(__nv_bfloat16));
   w.partial = reinterpret_cast<float*>(base ? base + off : nullptr);
-  off = up(off + (size_t)shrink_splits(T, d_in) * T * R * sizeof(float));
+  if (splits > 1) off = up(off + (size_t)splits * T * R * sizeof(float));
+  w.counters = reinterpret_cast<int*>(base ? base + off : nullptr);
+  w.flags = w.counters + n_m;
+  w.sync_bytes = sizeof(int) * 2 * (size_t)n_m;
+  off = up(off + w.sync_bytes);
   return off;
 }
 
@@ -570,54 +663,56 @@ extern "C" cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64
   if (ldx % 8 != 0 || ldw % 8 != 0 || ldy % 8 != 0 || (adapter && (lda % 8 != 0 || ldb % 8 != 0))) return CWL_ERR_SHAPE;
   if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || (adapter && (!aligned16(A) || !aligned16(B))))
     return CWL_ERR_SHAPE;
-  if (T == 0) return CWL_OK;
   if (adapter && (table.offsets == nullptr || table.rank == nullptr || table.scale == nullptr ||
                   table.flags == nullptr || table.n_chunks == nullptr || table.capacity < 0))
     return CWL_ERR_INVALID_ARG;
+  if (T == 0) return CWL_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
 
-  ApplyWorkspace ws{nullptr, nullptr};
+  ApplyWorkspace ws{nullptr, nullptr, nullptr, nullptr, 0};
   if (adapter) {
     const size_t need = carve_apply(ws, static_cast<char*>(workspace), T, d_in, R);
     if (workspace == nullptr || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
       return CWL_ERR_WORKSPACE;
   }
 
-  CUtensorMap mX, mW, mH, mB, mA;
+  CUtensorMap mX, mW, mA, mH, mB;
   if (!make_map(&mX, X, (uint64_t)d_in, (uint64_t)T, (uint64_t)ldx, BK, BM)) return CWL_ERR_CUDA;
   if (!make_map(&mW, W, (uint64_t)d_out, (uint64_t)d_in, (uint64_t)ldw, 64, BK)) return CWL_ERR_CUDA;
-
   if (adapter) {
     if (!make_map(&mA, A, (uint64_t)R, (uint64_t)d_in, (uint64_t)lda, 64, BK)) return CWL_ERR_CUDA;
     if (!make_map(&mH, ws.Hg, (uint64_t)R, (uint64_t)T, (uint64_t)R, BK, BM)) return CWL_ERR_CUDA;
     if (!make_map(&mB, B, (uint64_t)d_out, (uint64_t)R, (uint64_t)ldb, 64, BK)) return CWL_ERR_CUDA;
-
-    // 1. shrink: partial[s] = X[:, split s of d_in] A[split s, :]
-    GemmParams sp{};
-    sp.M = T; sp.N = R; sp.K0 = d_in; sp.K1 = 0;
-    sp.n_m_tiles = ceil_div(T, BM); sp.n_n_tiles = 1;
-    sp.splits = shrink_splits(T, d_in);
-    sp.kb_per_split = ceil_div(ceil_div(d_in, BK), sp.splits);
-    sp.out = ws.partial; sp.ld_out = R; sp.status_word = status_word;
-    cwl_status st;
-    if (R <= 64)       st = launch_gemm<64, 6, MODE_SHRINK>(mX, mA, mX, mA, sp, stream);
-    else if (R <= 128) st = launch_gemm<128, 6, MODE_SHRINK>(mX, mA, mX, mA, sp, stream);
-    else               st = launch_gemm<256, 4, MODE_SHRINK>(mX, mA, mX, mA, sp, stream);
-    if (st != CWL_OK) return st;
-
-    // 2. gate
-    gate_kernel<<<ceil_div(T, kGateRows), kGateThreads, 0, stream>>>(ws.partial, sp.splits, T, R, table, window, ws.Hg);
-    CWL_CUDA_TRY(cudaGetLastError());
+  } else {
+    mA = mW; mH = mX; mB = mW;   // never dereferenced when R == 0
   }
 
-  // 3. project: Y = [X | H'] [W ; B]
-  GemmParams gp{};
-  gp.M = T; gp.N = d_out; gp.K0 = d_in; gp.K1 = adapter ? R : 0;
-  gp.n_m_tiles = ceil_div(T, BM); gp.n_n_tiles = ceil_div(d_out, 256);
-  gp.splits = 1; gp.kb_per_split = ceil_div(d_in, BK);
-  gp.out = Y; gp.ld_out = ldy; gp.status_word = status_word;
-  if (adapter) return launch_gemm<256, 4, MODE_PROJECT>(mX, mW, mH, mB, gp, stream);
-  return launch_gemm<256, 4, MODE_PROJECT>(mX, mW, mX, mW, gp, stream);
+  ApplyParams p{};
+  p.T = T; p.d_in = d_in; p.d_out = d_out; p.R = adapter ? R : 0;
+  p.r_pad = adapter ? ceil_div(R, 64) * 64 : 0;
+  p.n_m_tiles = ceil_div(T, BM); p.n_n_tiles = ceil_div(d_out, BN);
+  p.splits = adapter ? shrink_splits(T, d_in) : 1;
+  p.kb_per_split = ceil_div(ceil_div(d_in, BK), p.splits);
+  p.window = window;
+  p.Y = static_cast<__nv_bfloat16*>(Y); p.ldy = ldy;
+  p.Hg = ws.Hg; p.partial = ws.partial; p.counters = ws.counters; p.flags = ws.flags;
+  p.table = table; p.status_word = status_word;
+
+  // the per-row-tile counters and flags are the only words that must start at zero
+  if (adapter) CWL_CUDA_TRY(cudaMemsetAsync(ws.counters, 0, ws.sync_bytes, stream));
+
+  static bool configured[64] = {};  // per device; benign race: the attribute call is idempotent
+  int dev = 0;
+  CWL_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
+    CWL_CUDA_TRY(cudaFuncSetAttribute(apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemPlan::kTotal));
+    if (dev >= 0 && dev < 64) configured[dev] = true;
+  }
+  const int items = p.n_m_tiles * p.n_n_tiles;
+  const int grid = items < sm_count() ? items : sm_count();
+  apply_kernel<<<grid, kGemmThreads, SmemPlan::kTotal, stream>>>(mX, mW, mA, mH, mB, p);
+  CWL_CUDA_TRY(cudaGetLastError());
+  return CWL_OK;
 }
 
 // ------------------------------------------------------------------------------ no-allocation variant

@@ -48,7 +48,7 @@ def test_matches_cwl_apply_on_two_calls_in_a_row():
 
 
 def test_rejects_problems_larger_than_the_built_in_scratch():
-    T, d_in, R = 16384, 4096, 64
+    T, d_in, R = 16384, 1024, 256
     assert cwl.cwl_apply_workspace_bytes(T, d_in, 256, R) > cwl.NOALLOC_SCRATCH_BYTES
     X = torch.zeros(T, d_in, dtype=torch.bfloat16, device="cuda")
     W = torch.zeros(d_in, 256, dtype=torch.bfloat16, device="cuda")
