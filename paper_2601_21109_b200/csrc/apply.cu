@@ -3,7 +3,11 @@
 //   y_t = x_t W + ((x_t A) * g_t) B,   g_t[j] = (1-lam_t) s_p [j < r_p] + lam_t s_c [j < r_c]
 //
 // which, by linearity, equals blending the outgoing and incoming adapter outputs.  ONE persistent,
-// warp-specialised kernel does all of it.  Each CTA first works through its share of SHRINK items
+// warp-specialised kernel does all of it, launched as clusters of two CTAs: a pair owns 256 rows and
+// issues tcgen05.mma with cta_group::2, so each CTA stages only its 128 rows of the left operand and
+// HALF of the right operand per pipeline step (a third less shared-memory fill per FLOP than a
+// single-CTA 128 x 256 tile, which is what bounded the single-CTA version).
+// Each pair first works through its share of SHRINK items
 //   P[split] = X[:, split of d_in] A[split, :]   (full ladder rank R, fp32 partials when d_in is split),
 // the CTA that completes a row tile's last split sums the partials, applies the per-row gate (rank
 // mask, scale and cross-fade weight from the chunk table, expanded per row in shared memory) and
@@ -12,9 +16,11 @@
 // whose K loop runs over d_in and then over R into ONE TMEM accumulator (the TMA producer acquires the
 // row tile's flag before its first H' load, ~d_in/64 pipeline steps after the tile began).
 //
-// Roles: warp 0 = TMA producer (cp.async.bulk.tensor, 128-byte swizzle), warp 1 = tcgen05.mma issuer
-// (cta_group::1, 128 x N x 16, bf16 -> fp32 in TMEM), warps 2..5 = epilogue (tcgen05.ld).  TMEM holds
-// two accumulators so the epilogue of one item overlaps the main loop of the next.  The left operand
+// Roles per CTA: warp 0 = TMA producer (cp.async.bulk.tensor, 128-byte swizzle, bytes counted on the
+// leader's mbarrier), warp 1 = tcgen05.mma issuer in the leader CTA only (256 x N x 16 across the pair,
+// bf16 -> fp32 in TMEM; tcgen05.commit multicast frees the stage in both CTAs), warps 2..5 = epilogue
+// (tcgen05.ld of the CTA's own 128 accumulator rows).  TMEM holds two accumulators so the epilogue of
+// one item overlaps the main loop of the next.  The left operand
 // is K-major (rows of X / H'), the right operand is N-major (rows of W, A, B are contiguous in their
 // output dimension), exactly as the matrices sit in HBM.
 //
@@ -23,6 +29,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <cstdio>
+#include <cstdlib>
 #include <mutex>
 #include <unordered_map>
 
@@ -35,11 +43,15 @@ constexpr int BM = 128;             // rows per tile = TMEM lanes
 constexpr int BN = 256;             // columns per projection tile = one TMEM accumulator
 constexpr int BK = 64;              // K elements per stage = one 128-byte swizzle row of bf16
 constexpr int UMMA_K = 16;
-constexpr int kStages = 4;
+#ifndef CWL_STAGES
+#define CWL_STAGES 6
+#endif
+constexpr int kStages = CWL_STAGES;
 constexpr int kGemmThreads = 192;   // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
 constexpr int kEpilogueThreads = 128;
-constexpr int kGroupM = 16;         // row tiles per raster group (keeps their X rows L2-resident)
+constexpr int kGroupM = 8;          // pair rows (256 tokens each) per raster group: their X rows stay L2-resident
 constexpr int kNumSmsPlanned = 148; // used where the answer must not depend on the device
+constexpr int kPairsPlanned = kNumSmsPlanned / 2;
 constexpr int kMaxSplits = 16;      // split factor of the shrink along d_in
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
@@ -47,15 +59,15 @@ struct RowGate { float w_in, w_out; int r_in, r_out; };  // g[j] = w_in [j < r_i
 
 struct ApplyParams {
   int T, d_in, d_out, R;   // R = 0: no adapter
-  int r_pad;               // R rounded up to the 64-column swizzle atom
-  int n_m_tiles, n_n_tiles;
+  int r_pad;               // R rounded up to 128: each CTA of a pair supplies whole 64-column swizzle atoms
+  int n_m_pairs, n_n_tiles;
   int splits, kb_per_split;
   int window;
   __nv_bfloat16* Y; int64_t ldy;
   __nv_bfloat16* Hg;       // [T, R] gated shrink output
   float* partial;          // [splits, T, R]
-  int* counters;           // [n_m_tiles] splits finished per row tile
-  int* flags;              // [n_m_tiles] 1 once H' of the row tile is published
+  int* counters;           // [2 n_m_pairs] splits finished per 128-row tile
+  int* flags;              // [2 n_m_pairs] 1 once H' of the 128-row tile is published
   cwl_chunk_table table;
   int32_t* status_word;
 };
@@ -99,10 +111,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+// TMA load into THIS CTA's shared memory whose bytes are counted on the pair leader's mbarrier
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t leader_bar, int x, int y) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(leader_bar), "r"(x), "r"(y) : "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -112,26 +125,29 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
 }
 __device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem], 128 x N x 16, bf16 in, fp32 out
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
+// D[tmem] (+)= A[smem] * B[smem] across the CTA pair: 256 x N x 16, bf16 in, fp32 out.  Each CTA supplies its
+// 128 rows of A and its half of B's columns, and receives its 128 rows of D in its own TMEM.
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
-// mbarrier arrives once every MMA issued so far by this thread has finished
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// the mbarrier at this shared-memory offset arrives in BOTH CTAs once every MMA issued so far has finished
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t both = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(both) : "memory");
 }
 // 32 consecutive fp32 columns of this thread's TMEM lane
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -184,42 +200,61 @@ __device__ __forceinline__ void st_release(int* p, int v) {
 // orders this thread's generic-proxy observations before its later async-proxy (TMA) accesses
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in CTA `cta` of the cluster
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t cta) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(cta));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+
 // ------------------------------------------------------------------------------------ work items
 enum : int { ITEM_SHRINK = 0, ITEM_PROJECT = 1 };
-struct Item { int kind, m_tile, n_tile, split; };
+struct Item { int kind, m_pair, n_tile, split; };
 
 struct SmemPlan {
-  static constexpr int kABytes = BM * BK * 2;       // 16 KB: one TMA box of X or H'
-  static constexpr int kBBytes = BN * BK * 2;       // 32 KB: four 64 x 64 boxes of W, B or A
+  static constexpr int kABytes = BM * BK * 2;        // 16 KB: one TMA box of X or H' (this CTA's 128 rows)
+  static constexpr int kBBytes = (BN / 2) * BK * 2;  // 16 KB: this CTA's half of the right operand (two 64 x 64 boxes)
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kTileBytes = kStages * kStageBytes;
   static constexpr int kBarBytes = (2 * kStages + 4) * 8;
-  static constexpr int kMiscBytes = 32;             // TMEM base, abort flag, epilogue broadcast words
+  static constexpr int kMiscBytes = 32;              // TMEM base, abort flag, epilogue broadcast words
   static constexpr int kGateBytes = BM * (int)sizeof(RowGate);
   static constexpr int kTotal = kTileBytes + kBarBytes + kMiscBytes + kGateBytes + 1024;  // + alignment slack
 };
 
-// The i-th work item of this CTA.  Shrink items come first and are dealt from the LAST CTA downwards,
-// so the CTAs that receive one projection tile fewer carry the shrink work.  Projection tiles are
-// rastered in groups of kGroupM row tiles (row tile fastest inside a group).
+// The i-th work item of this CTA pair.  A pair owns 256 rows (CTA rank r the rows 128 r .. 128 r + 127).
+// Shrink items come first and are dealt from the LAST pair downwards, so the pairs that receive one
+// projection tile fewer carry the shrink work.  Projection tiles are rastered in groups of kGroupM pair
+// rows (pair row fastest inside a group) so a group's X rows and the W column slabs stay in L2.
 __device__ __forceinline__ bool get_item(int i, const ApplyParams& p, Item& it) {
-  const int G = gridDim.x, b = blockIdx.x;
-  const int n_shrink = (p.R > 0) ? p.n_m_tiles * p.splits : 0;
+  const int G = gridDim.x >> 1, b = blockIdx.x >> 1;
+  const int n_shrink = (p.R > 0) ? p.n_m_pairs * p.splits : 0;
   const int first_s = G - 1 - b;
   const int my_shrink = first_s < n_shrink ? (n_shrink - 1 - first_s) / G + 1 : 0;
   if (i < my_shrink) {
     const int s = first_s + i * G;
-    it.kind = ITEM_SHRINK; it.m_tile = s / p.splits; it.split = s - it.m_tile * p.splits; it.n_tile = 0;
+    it.kind = ITEM_SHRINK; it.m_pair = s / p.splits; it.split = s - it.m_pair * p.splits; it.n_tile = 0;
     return true;
   }
   const int tile = b + (i - my_shrink) * G;
-  if (tile >= p.n_m_tiles * p.n_n_tiles) return false;
+  if (tile >= p.n_m_pairs * p.n_n_tiles) return false;
   const int per_group = kGroupM * p.n_n_tiles;
   const int group = tile / per_group, within = tile - group * per_group;
   const int first_m = group * kGroupM;
-  const int gsize = min(kGroupM, p.n_m_tiles - first_m);
+  const int gsize = min(kGroupM, p.n_m_pairs - first_m);
   it.kind = ITEM_PROJECT; it.split = 0;
-  it.m_tile = first_m + within % gsize;
+  it.m_pair = first_m + within % gsize;
   it.n_tile = within / gsize;
   return true;
 }
@@ -277,7 +312,7 @@ __device__ __forceinline__ bool wait_flag(const int* flag, volatile int* abort_f
   }
 }
 
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
              const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_h,
              const __grid_constant__ CUtensorMap tm_b, const ApplyParams p) {
@@ -301,10 +336,14 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
   RowGate* gates = reinterpret_cast<RowGate*>(misc + Plan::kMiscBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair (issues the MMAs)
 
   if (threadIdx.x == 0) {
+    // full: armed by the leader's producer, completed by both CTAs' TMA bytes (only the leader's copy is used)
+    // empty / acc_full: one arrival from the leader's tcgen05.commit, multicast to both CTAs
+    // acc_empty: the 128 epilogue threads of BOTH CTAs arrive on the leader's copy
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), kEpilogueThreads); }
+    for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 2 * kEpilogueThreads); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tmap(&tm_x);
@@ -317,11 +356,12 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
   }
   tc_fence_before();
   __syncthreads();
+  cluster_sync();                                   // the peer's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
     if (lane == 0) {
       uint32_t it_cnt = 0;      // running stage counter across items
       bool ok = true;
@@ -330,31 +370,34 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         int kb0, n0, n1;
         item_blocks(item, p, kb0, n0, n1);
         const bool shrink = item.kind == ITEM_SHRINK;
-        const int n_boxes = shrink ? p.r_pad / 64 : BN / 64;
-        const uint32_t tx = Plan::kABytes + n_boxes * (BK * 128);
+        const int m_tile = item.m_pair * 2 + (int)rank;       // this CTA's 128-row tile
+        const int half = shrink ? p.r_pad / 2 : BN / 2;       // columns of the right operand this CTA supplies
+        const int n_boxes = half / 64;
+        const uint32_t tx_pair = 2u * (Plan::kABytes + n_boxes * (BK * 128));
         const CUtensorMap* right0 = shrink ? &tm_a : &tm_w;
-        const int col0 = shrink ? 0 : item.n_tile * BN;
+        const int col0 = (shrink ? 0 : item.n_tile * BN) + (int)rank * half;
         for (int b = 0; b < n0 + n1; ++b, ++it_cnt) {
           const int s = it_cnt % kStages;
           const uint32_t ph = (it_cnt / kStages) & 1u;
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
           const bool phase1 = b >= n0;
           if (phase1 && b == n0) {
-            // H' of this row tile must have been published by whoever finished its shrink
-            if (!wait_flag(p.flags + item.m_tile, abort_flag)) { ok = false; break; }
+            // H' of this CTA's row tile must have been published by whoever finished its shrink
+            if (!wait_flag(p.flags + m_tile, abort_flag)) { ok = false; break; }
             fence_proxy_async();
           }
           const int k = phase1 ? (b - n0) * BK : (kb0 + b) * BK;
           const CUtensorMap* left = phase1 ? &tm_h : &tm_x;
           const CUtensorMap* right = phase1 ? &tm_b : right0;
           const uint32_t sa = base + s * Plan::kStageBytes, sb = sa + Plan::kABytes;
-          mbar_expect_tx(full_bar(s), tx);
-          tma_load_2d(sa, left, full_bar(s), k, item.m_tile * BM);
+          const uint32_t leader_full = full_bar(s) & 0xFEFFFFFFu;   // the same barrier in the leader's shared memory
+          if (rank == 0) mbar_expect_tx(full_bar(s), tx_pair);
+          tma_load_2d_pair(sa, left, leader_full, k, m_tile * BM);
           for (int j = 0; j < n_boxes; ++j)
-            tma_load_2d(sb + j * (BK * 128), right, full_bar(s), col0 + j * 64, k);
+            tma_load_2d_pair(sb + j * (BK * 128), right, leader_full, col0 + j * 64, k);
         }
       }
-      if (!ok) {
+      if (!ok && rank == 0) {
         // drain: give the copies already issued a bounded chance to land before the CTA leaves
         for (uint32_t back = 1; back <= (uint32_t)kStages && back <= it_cnt; ++back) {
           const uint32_t j = it_cnt - back;
@@ -364,10 +407,10 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc_project = make_idesc(BM, BN);
-      const uint32_t idesc_shrink = make_idesc(BM, p.r_pad > 0 ? p.r_pad : 64);
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc_project = make_idesc(2 * BM, BN);
+      const uint32_t idesc_shrink = make_idesc(2 * BM, p.r_pad > 0 ? p.r_pad : 128);
       uint32_t it_cnt = 0, local = 0;
       bool ok = true;
       Item item;
@@ -392,11 +435,11 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
           for (int kk = 0; kk < k_steps; ++kk) {
             const uint64_t da = make_smem_desc(sa + kk * (UMMA_K * 2), 16, 1024);
             const uint64_t db = make_smem_desc(sb + kk * (UMMA_K * 128), BK * 128, 1024);
-            umma_bf16(d_tmem, da, db, idesc, (b | kk) != 0 ? 1u : 0u);
+            umma_bf16_pair(d_tmem, da, db, idesc, (b | kk) != 0 ? 1u : 0u);
           }
-          umma_commit(empty_bar(s));            // frees the stage once these MMAs have read it
+          umma_commit_pair(empty_bar(s));            // frees the stage in both CTAs once these MMAs have read it
         }
-        if (ok) umma_commit(acc_full_bar(acc)); // accumulator complete
+        if (ok) umma_commit_pair(acc_full_bar(acc)); // accumulator complete, both CTAs
       }
       if (!ok) {
         // give the MMAs still in flight a bounded time to retire before TMEM is released
@@ -405,7 +448,7 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
     const int lane_group = warp & 3;              // TMEM lanes this warp may read: 32*lane_group ..
     const int row_in_tile = lane_group * 32 + lane;
     const int epi_tid = threadIdx.x - 64;         // 0..127
@@ -420,8 +463,10 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       epilogue_barrier();
       if (*epi_go == 0) break;
       tc_fence_after();
-      const int row = item.m_tile * BM + row_in_tile;
+      const int m_tile = item.m_pair * 2 + (int)rank;
+      const int row = m_tile * BM + row_in_tile;
       const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(lane_group * 32) << 16);
+      const uint32_t leader_acc_empty = mapa_shared(acc_empty_bar(acc), 0);
 
       if (item.kind == ITEM_PROJECT) {
 #pragma unroll 1
@@ -447,7 +492,7 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
           }
         }
         tc_fence_before();
-        mbar_arrive(acc_empty_bar(acc));
+        mbar_arrive_cluster(leader_acc_empty);
         continue;
       }
 
@@ -488,26 +533,26 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         }
       }
       tc_fence_before();
-      mbar_arrive(acc_empty_bar(acc));               // the accumulator is free again
+      mbar_arrive_cluster(leader_acc_empty);         // the accumulator is free again
 
       __threadfence();                               // this thread's H' / partial stores, device-wide
       epilogue_barrier();
       if (direct) {
-        if (epi_tid == 0) st_release(p.flags + item.m_tile, 1);
+        if (epi_tid == 0) st_release(p.flags + m_tile, 1);
         continue;
       }
-      if (epi_tid == 0) *epi_last = (atomicAdd(p.counters + item.m_tile, 1) == p.splits - 1);
+      if (epi_tid == 0) *epi_last = (atomicAdd(p.counters + m_tile, 1) == p.splits - 1);
       epilogue_barrier();
       if (*epi_last == 0) continue;
-      // this CTA completed the row tile: sum the partials, gate, publish H'
+      // this CTA completed its row tile: sum the partials, gate, publish H'
       __threadfence();
-      gates[epi_tid] = row_gate(item.m_tile * BM + epi_tid, p);
+      gates[epi_tid] = row_gate(m_tile * BM + epi_tid, p);
       epilogue_barrier();
       const int quads = p.R >> 2;                    // float4 groups per row
       const int64_t split_stride = (int64_t)p.T * p.R;
       for (int idx = epi_tid; idx < BM * quads; idx += kEpilogueThreads) {
         const int r = idx / quads, j0 = (idx - r * quads) << 2;
-        const int t = item.m_tile * BM + r;
+        const int t = m_tile * BM + r;
         if (t >= p.T) break;
         const RowGate gr = gates[r];
         float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -523,13 +568,14 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       }
       __threadfence();
       epilogue_barrier();
-      if (epi_tid == 0) st_release(p.flags + item.m_tile, 1);
+      if (epi_tid == 0) st_release(p.flags + m_tile, 1);
     }
   }
 
   // ---------------------------------------------------------------------- teardown
   tc_fence_before();
   __syncthreads();
+  cluster_sync();   // neither CTA leaves (or frees TMEM) while the other may still signal it or write its TMEM
   if (threadIdx.x == 0 && *abort_flag) flag_status(p.status_word, CWL_ERR_TIMEOUT);
   if (warp == 1) {
     tc_fence_after();
@@ -608,10 +654,33 @@ int sm_count() {
   return n;
 }
 
+// CTA pairs that can be resident at once (clusters of 2 need both SMs in one GPC)
+int max_pairs() {
+  static int n = []() {
+    int v = 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * kPairsPlanned, 1, 1);
+    cfg.blockDim = dim3(kGemmThreads, 1, 1);
+    cfg.dynamicSmemBytes = SmemPlan::kTotal;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    if (cudaFuncSetAttribute(apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemPlan::kTotal) != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&v, apply_kernel, &cfg) != cudaSuccess || v <= 0) {
+      cudaGetLastError();
+      v = sm_count() / 2;
+    }
+    if (getenv("CWL_LOG") != nullptr) fprintf(stderr, "[cwl] resident CTA pairs: %d (SMs %d)\n", v, sm_count());
+    return v;
+  }();
+  return n;
+}
+
 // split factor of the shrink along d_in: enough items to spread X over the SMs when T is small
 int shrink_splits(int T, int d_in) {
-  const int n_m = ceil_div(T, BM), nkb = ceil_div(d_in, BK);
-  int s = kNumSmsPlanned / n_m;
+  const int n_pairs = ceil_div(T, 2 * BM), nkb = ceil_div(d_in, BK);
+  int s = kPairsPlanned / n_pairs;
   if (s > kMaxSplits) s = kMaxSplits;
   if (s > nkb) s = nkb;
   if (s < 1) s = 1;
@@ -623,7 +692,7 @@ struct ApplyWorkspace { __nv_bfloat16* Hg; float* partial; int* counters; int* f
 
 size_t carve_apply(ApplyWorkspace& w, char* base, int T, int d_in, int R) {
   auto up = [](size_t x) { return (x + 255) / 256 * 256; };
-  const int splits = shrink_splits(T, d_in), n_m = ceil_div(T, BM);
+  const int splits = shrink_splits(T, d_in), n_m = 2 * ceil_div(T, 2 * BM);
   size_t off = 0;
   w.Hg = reinterpret_cast<__nv_bfloat16*>(base ? base + off : nullptr);
   off = up(off + (size_t)T * R * sizeof(__nv_bfloat16));
@@ -689,8 +758,8 @@ extern "C" cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64
 
   ApplyParams p{};
   p.T = T; p.d_in = d_in; p.d_out = d_out; p.R = adapter ? R : 0;
-  p.r_pad = adapter ? ceil_div(R, 64) * 64 : 0;
-  p.n_m_tiles = ceil_div(T, BM); p.n_n_tiles = ceil_div(d_out, BN);
+  p.r_pad = adapter ? ceil_div(R, 128) * 128 : 0;
+  p.n_m_pairs = ceil_div(T, 2 * BM); p.n_n_tiles = ceil_div(d_out, BN);
   p.splits = adapter ? shrink_splits(T, d_in) : 1;
   p.kb_per_split = ceil_div(ceil_div(d_in, BK), p.splits);
   p.window = window;
@@ -708,9 +777,9 @@ extern "C" cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64
     CWL_CUDA_TRY(cudaFuncSetAttribute(apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemPlan::kTotal));
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
-  const int items = p.n_m_tiles * p.n_n_tiles;
-  const int grid = items < sm_count() ? items : sm_count();
-  apply_kernel<<<grid, kGemmThreads, SmemPlan::kTotal, stream>>>(mX, mW, mA, mH, mB, p);
+  const int items = p.n_m_pairs * p.n_n_tiles, pairs_max = max_pairs();
+  const int pairs = items < pairs_max ? items : pairs_max;
+  apply_kernel<<<2 * pairs, kGemmThreads, SmemPlan::kTotal, stream>>>(mX, mW, mA, mH, mB, p);
   CWL_CUDA_TRY(cudaGetLastError());
   return CWL_OK;
 }
