@@ -57,7 +57,8 @@ constexpr int kBoxCols = 64;        // columns of one right-operand TMA box (one
 constexpr int kABytes = BM * BK * 2;          // 16 KB: this CTA's 128 rows of the left operand
 constexpr int kBoxBytes = kBoxCols * BK * 2;  // 8 KB
 constexpr int kMaxStages = 8;
-constexpr int kRingBytes = 208 * 1024;
+constexpr int kRingBytes = 192 * 1024;
+constexpr int kOutBufBytes = 4096;  // per epilogue warp: 32 rows x 64 bf16 columns staged for a TMA store
 constexpr int kThreads = 320;       // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: epilogue
 constexpr int kEpiThreads = 256;
 constexpr int kEpiWarps = 8;
@@ -88,7 +89,7 @@ struct ApplyParams {
   int window;
   __nv_bfloat16* Y; int64_t ldy;
   __nv_bfloat16* Hg;       // [T, R] gated shrink output
-  float* partial;          // [shrink_splits, T, R]
+  float* partial;          // [shrink_splits, 128-row tiles, R / 4, 128, 4] fp32 partial shrink sums
   float* sk_partial;       // [tiles * split_k * 2, 128, w0] fp32 partial accumulators of split-K items
   int* counters;           // [2 n_m_pairs] shrink splits finished per 128-row tile
   int* flags;              // [2 n_m_pairs] 1 once H' of the 128-row tile is published
@@ -139,6 +140,17 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
   asm volatile(
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(map), "r"(leader_bar), "r"(x), "r"(y) : "memory");
+}
+// TMA store of a staged box (shared -> global); rows and columns outside the tensor are clipped
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -348,16 +360,19 @@ __device__ __forceinline__ bool wait_word(const int* word, int target, volatile 
 }
 
 struct SmemLayout {
+  static constexpr int kOutBytes = kEpiWarps * kOutBufBytes;   // also holds the row gates of a shrink finaliser
   static constexpr int kBarBytes = (2 * kMaxStages + 2) * 8;
   static constexpr int kMiscBytes = 32;              // TMEM base, abort flag, epilogue broadcast words
-  static constexpr int kGateBytes = BM * (int)sizeof(RowGate);
-  static constexpr int kTotal = kRingBytes + kBarBytes + kMiscBytes + kGateBytes + 1024;  // + alignment slack
+  static constexpr int kTotal = kRingBytes + kOutBytes + kBarBytes + kMiscBytes + 1024;  // + alignment slack
 };
+static_assert(BM * sizeof(RowGate) <= SmemLayout::kOutBytes, "row gates must fit the staging area");
+static_assert(SmemLayout::kTotal <= 227 * 1024, "shared memory budget");
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
              const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_h,
-             const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ ApplyParams p) {
+             const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_y,
+             const __grid_constant__ ApplyParams p) {
   using L = SmemLayout;
   constexpr uint32_t kTmemCols = kMaxTileW;
 
@@ -365,17 +380,18 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;     // swizzled tiles need 1024-byte alignment
   uint8_t* base_ptr = smem_raw + (base - raw);
-  const uint32_t bars = base + kRingBytes;
+  const uint32_t out_bufs = base + kRingBytes;      // 1024-byte aligned: the TMA store reads it with the 128-byte swizzle
+  const uint32_t bars = out_bufs + L::kOutBytes;
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
   const uint32_t acc_full_bar = bars + 8u * (2 * kMaxStages);
   const uint32_t acc_empty_bar = bars + 8u * (2 * kMaxStages + 1);
-  uint8_t* misc = base_ptr + kRingBytes + L::kBarBytes;
+  uint8_t* misc = base_ptr + kRingBytes + L::kOutBytes + L::kBarBytes;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
   volatile int* epi_go = reinterpret_cast<volatile int*>(misc + 8);     // epilogue: proceed with this item?
   volatile int* epi_last = reinterpret_cast<volatile int*>(misc + 12);  // epilogue: this CTA finalises the row tile
-  RowGate* gates = reinterpret_cast<RowGate*>(misc + L::kMiscBytes);
+  RowGate* gates = reinterpret_cast<RowGate*>(base_ptr + kRingBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair (issues the MMAs)
@@ -395,6 +411,7 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tmap(&tm_x);
     prefetch_tmap(&tm_w);
+    prefetch_tmap(&tm_y);
     if (p.R > 0) { prefetch_tmap(&tm_a); prefetch_tmap(&tm_h); prefetch_tmap(&tm_b); }
   }
   if (warp == 1) {
@@ -524,26 +541,35 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       const int n_chunks = (item.wt + 31) >> 5;
 
       if (item.kind == ITEM_PROJECT && pl.split_k == 1) {
-        // ---- whole tile: accumulator -> bf16 -> Y ----
+        // ---- whole tile: accumulator -> bf16 -> swizzled staging buffer -> TMA store of 32 x 64 boxes ----
+        const uint32_t obuf = out_bufs + (uint32_t)(warp - 2) * kOutBufBytes;
+        const int n64 = (item.wt + 63) >> 6;         // a ragged width only occurs at the edge of Y: the store clips it
+        const int row0 = m_tile * BM + quad * 32;
 #pragma unroll 1
-        for (int cc = chalf; cc < n_chunks; cc += 2) {
-          const int col = item.n0 + cc * 32;
-          uint32_t v[32];
-          tmem_ld32(t_row + cc * 32, v);
-          tmem_ld_wait();
-          if (row < p.T) {
-            __nv_bfloat16* out = p.Y + (int64_t)row * p.ldy + col;
+        for (int c64 = chalf; c64 < n64; c64 += 2) {
+          if (lane == 0) bulk_wait_read();           // the previous store has finished reading this buffer
+          __syncwarp();
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            uint32_t v[32];
+            tmem_ld32(t_row + c64 * 64 + h * 32, v);
+            tmem_ld_wait();
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
-              if (cc * 32 + g * 8 < item.wt) {       // widths are multiples of 8: a granule is all in or all out
-                uint4 q;
-                q.x = pack_bf16(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
-                q.y = pack_bf16(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
-                q.z = pack_bf16(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5]));
-                q.w = pack_bf16(__uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7]));
-                *reinterpret_cast<uint4*>(out + g * 8) = q;
-              }
+              uint4 q;
+              q.x = pack_bf16(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
+              q.y = pack_bf16(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
+              q.z = pack_bf16(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5]));
+              q.w = pack_bf16(__uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7]));
+              const int piece = h * 4 + g;           // 16-byte piece of this lane's 128-byte row
+              st_shared_v4(obuf + lane * 128 + ((piece ^ (lane & 7)) << 4), q);
             }
+          }
+          fence_proxy_async();                       // the staged rows, visible to the TMA engine
+          __syncwarp();
+          if (lane == 0 && row0 < p.T) {
+            tma_store_2d(&tm_y, obuf, item.n0 + c64 * 64, row0);
+            bulk_commit();
           }
         }
         tc_fence_before();
@@ -554,17 +580,18 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
 
       if (item.kind == ITEM_PROJECT) {
         // ---- split-K item: store the fp32 partial, then reduce this item's share of the tile's columns ----
+        // partial layout [column group of 4][128 rows][4]: a warp's store and the reducer's loads are contiguous
         float* mine = p.sk_partial + ((int64_t)(item.tile * pl.split_k + item.split) * 2 + rank) * (BM * pl.w0);
 #pragma unroll 1
         for (int cc = chalf; cc < n_chunks; cc += 2) {
           uint32_t v[32];
           tmem_ld32(t_row + cc * 32, v);
           tmem_ld_wait();
-          float* out = mine + row_in_tile * pl.w0 + cc * 32;
 #pragma unroll
           for (int q4 = 0; q4 < 8; ++q4)
             if (cc * 32 + q4 * 4 < item.wt)
-              *reinterpret_cast<uint4*>(out + q4 * 4) = make_uint4(v[q4 * 4 + 0], v[q4 * 4 + 1], v[q4 * 4 + 2], v[q4 * 4 + 3]);
+              *reinterpret_cast<uint4*>(mine + ((cc * 8 + q4) * BM + row_in_tile) * 4) =
+                  make_uint4(v[q4 * 4 + 0], v[q4 * 4 + 1], v[q4 * 4 + 2], v[q4 * 4 + 3]);
         }
         tc_fence_before();
         __syncwarp();
@@ -579,18 +606,20 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         epilogue_barrier();
         if (*epi_go == 0) break;
         __threadfence();
-        // columns [c_lo, c_hi) of the tile are this item's to reduce (multiples of 8)
+        // columns [c_lo, c_hi) of the tile are this item's to reduce (multiples of 8).  This is the pair's last
+        // item and its MMAs have retired, so the operand ring is free: the bf16 result is staged there row by row
+        // and written to Y with contiguous 16-byte stores.
         const int share = (((item.wt + pl.split_k - 1) / pl.split_k) + 7) & ~7;
         const int c_lo = min(item.wt, item.split * share), c_hi = min(item.wt, c_lo + share);
-        const int quads = (c_hi - c_lo) >> 2;
+        const int n_cg = (c_hi - c_lo) >> 2;
+        const int pitch = share * 2 + 16;            // bytes per staged row
         const float* tile_base = p.sk_partial + ((int64_t)(item.tile * pl.split_k) * 2 + rank) * (BM * pl.w0);
         const int64_t split_stride = (int64_t)2 * BM * pl.w0;
-        for (int idx = epi_tid; idx < BM * quads; idx += kEpiThreads) {
-          const int r = idx / quads, j0 = c_lo + ((idx - r * quads) << 2);
-          const int t = m_tile * BM + r;
-          if (t >= p.T) break;
+        for (int idx = epi_tid; idx < BM * n_cg; idx += kEpiThreads) {
+          const int r = idx & (BM - 1), cg = idx >> 7;
+          const float* src = tile_base + ((int64_t)((c_lo >> 2) + cg) * BM + r) * 4;
           float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-          const float* src = tile_base + r * pl.w0 + j0;
+#pragma unroll 4
           for (int s = 0; s < pl.split_k; ++s) {
             const float4 x = __ldcg(reinterpret_cast<const float4*>(src + s * split_stride));
             sum.x += x.x; sum.y += x.y; sum.z += x.z; sum.w += x.w;
@@ -598,7 +627,16 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
           uint2 o;
           o.x = pack_bf16(sum.x, sum.y);
           o.y = pack_bf16(sum.z, sum.w);
-          *reinterpret_cast<uint2*>(p.Y + (int64_t)t * p.ldy + item.n0 + j0) = o;
+          *reinterpret_cast<uint2*>(base_ptr + r * pitch + cg * 8) = o;
+        }
+        epilogue_barrier();
+        const int pieces = (c_hi - c_lo) >> 3;       // 16-byte pieces per row
+        for (int idx = epi_tid; idx < BM * pieces; idx += kEpiThreads) {
+          const int r = idx / pieces, pc = idx - r * pieces;
+          const int t = m_tile * BM + r;
+          if (t >= p.T) break;
+          const uint4 q = *reinterpret_cast<const uint4*>(base_ptr + r * pitch + pc * 16);
+          *reinterpret_cast<uint4*>(p.Y + (int64_t)t * p.ldy + item.n0 + c_lo + pc * 8) = q;
         }
         continue;
       }
@@ -613,8 +651,16 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         uint32_t v[32];
         tmem_ld32(t_row + cc * 32, v);
         tmem_ld_wait();
-        if (row < p.T) {
-          if (direct) {
+        if (!direct) {
+          // partial layout [split][128-row tile][column group of 4][128 rows][4]: contiguous per warp store
+          float* out = p.partial + (((int64_t)(item.split * 2 * pl.n_m_pairs + m_tile) * (p.R >> 2) + cc * 8) * BM + row_in_tile) * 4;
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4) {
+            if (col + q4 * 4 < p.R)
+              *reinterpret_cast<uint4*>(out + q4 * BM * 4) = make_uint4(v[q4 * 4 + 0], v[q4 * 4 + 1], v[q4 * 4 + 2], v[q4 * 4 + 3]);
+          }
+        } else if (row < p.T) {
+          {
             __nv_bfloat16* out = p.Hg + (int64_t)row * p.R + col;
 #pragma unroll
             for (int q8 = 0; q8 < 4; ++q8) {
@@ -627,13 +673,6 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 q.w = pack_bf16(__uint_as_float(v[q8 * 8 + 6]) * gate_at(g, j + 6), __uint_as_float(v[q8 * 8 + 7]) * gate_at(g, j + 7));
                 *reinterpret_cast<uint4*>(out + q8 * 8) = q;
               }
-            }
-          } else {
-            float* out = p.partial + ((int64_t)item.split * p.T + row) * p.R + col;
-#pragma unroll
-            for (int q4 = 0; q4 < 8; ++q4) {
-              if (col + q4 * 4 < p.R)
-                *reinterpret_cast<uint4*>(out + q4 * 4) = make_uint4(v[q4 * 4 + 0], v[q4 * 4 + 1], v[q4 * 4 + 2], v[q4 * 4 + 3]);
             }
           }
         }
@@ -656,14 +695,15 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       if (epi_tid < BM) gates[epi_tid] = row_gate(m_tile * BM + epi_tid, p);
       epilogue_barrier();
       const int quads = p.R >> 2;                    // float4 groups per row
-      const int64_t split_stride = (int64_t)p.T * p.R;
+      const int64_t split_stride = (int64_t)2 * pl.n_m_pairs * p.R * BM;
       for (int idx = epi_tid; idx < BM * quads; idx += kEpiThreads) {
-        const int r = idx / quads, j0 = (idx - r * quads) << 2;
+        const int r = idx & (BM - 1), cg = idx >> 7, j0 = cg << 2;
         const int t = m_tile * BM + r;
-        if (t >= p.T) break;
+        if (t >= p.T) continue;
         const RowGate gr = gates[r];
         float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-        const float* src = p.partial + (int64_t)t * p.R + j0;
+        const float* src = p.partial + (((int64_t)m_tile * quads + cg) * BM + r) * 4;
+#pragma unroll 4
         for (int s = 0; s < pl.shrink_splits; ++s) {
           const float4 x = __ldcg(reinterpret_cast<const float4*>(src + s * split_stride));
           sum.x += x.x; sum.y += x.y; sum.z += x.z; sum.w += x.w;
@@ -677,6 +717,7 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       epilogue_barrier();
       if (epi_tid == 0) st_release(p.flags + m_tile, 1);
     }
+    if (lane == 0) bulk_wait_all();                  // this warp's TMA stores have left shared memory and landed
   }
 
   // ---------------------------------------------------------------------- teardown
@@ -789,23 +830,49 @@ Plan make_plan(int T, int d_in, int d_out, int R, int pairs, bool allow_split_k)
   pl.stages = kRingBytes / (kABytes + pl.boxes * kBoxBytes);
   if (pl.stages > kMaxStages) pl.stages = kMaxStages;
 
-  // ---- shrink items go, one at a time, to the pair with the lightest load so far
-  long long load[kPairsPlanned];
+  // ---- shrink: how finely d_in is split and who does the items.  Items go, one at a time, to the pair with
+  // the lightest load so far.  An item costs its K blocks (16 KB of rows + the boxes of A) plus a fixed
+  // start-up and hand-over term worth a few K blocks; H' must be there when the first tiles reach the end of
+  // their d_in loop, so shrink work that keeps a pair busy beyond that point counts as a stall for everybody.
+  long long base_load[kPairsPlanned], load[kPairsPlanned];
   const int NW = pl.n_m_pairs * pl.n_wide * pl.split_k, NN = pl.n_m_pairs * pl.n_narrow;
   const long long cost_w0 = tile_cost(pl.w0, pl.split_k > 1 ? pl.kb_per_ksplit + pl.nkb1 : kbt);
   for (int g = 0; g < pl.pairs; ++g)
-    load[g] = dealt(0, NW, pl.pairs, g) * cost_w0 + dealt(NW, NN, pl.pairs, g) * tile_cost(pl.w1, kbt);
+    base_load[g] = dealt(0, NW, pl.pairs, g) * cost_w0 + dealt(NW, NN, pl.pairs, g) * tile_cost(pl.w1, kbt);
+  long long best_total = -1;
   if (R > 0) {
-    const long long cs = (long long)pl.kb_per_split * (16 + 8 * boxes_for(R / 2)) + 24;
-    const int n_shrink = pl.n_m_pairs * pl.shrink_splits;
-    for (int i = 0; i < n_shrink; ++i) {
-      int at = pl.pairs - 1;
-      for (int g = pl.pairs - 1; g >= 0; --g)
-        if (load[g] < load[at]) at = g;
-      load[at] += cs;
-      pl.sh_count[at]++;
+    const long long first_tile = (long long)(pl.split_k > 1 ? pl.kb_per_ksplit : pl.nkb0) * (16 + 8 * tile_boxes(pl.w0));
+    for (int want = 1; want <= kMaxSplits; want *= 2) {
+      if (want > pl.nkb0) break;
+      const int per = ceil_div(pl.nkb0, want), splits = ceil_div(pl.nkb0, per);
+      const long long cs = (long long)per * (16 + 8 * boxes_for(R / 2)) + 176;
+      const int n_shrink = pl.n_m_pairs * splits;
+      uint16_t count[kPairsPlanned];
+      long long shrink_time[kPairsPlanned];
+      for (int g = 0; g < pl.pairs; ++g) { load[g] = base_load[g]; count[g] = 0; shrink_time[g] = 0; }
+      for (int i = 0; i < n_shrink; ++i) {
+        int at = pl.pairs - 1;
+        for (int g = pl.pairs - 1; g >= 0; --g)
+          if (load[g] < load[at]) at = g;
+        load[at] += cs; shrink_time[at] += cs; count[at]++;
+      }
+      long long worst = 0, latest = 0;
+      for (int g = 0; g < pl.pairs; ++g) {
+        if (load[g] > worst) worst = load[g];
+        if (shrink_time[g] > latest) latest = shrink_time[g];
+      }
+      const long long due = first_tile * 4 / 5;
+      const long long total = worst + (latest > due ? latest - due : 0);
+      if (best_total < 0 || total < best_total) {
+        best_total = total;
+        pl.shrink_splits = splits; pl.kb_per_split = per;
+        for (int g = 0; g < kPairsPlanned; ++g) pl.sh_count[g] = g < pl.pairs ? count[g] : 0;
+      }
     }
+    pl.makespan = best_total;
+    return pl;
   }
+  for (int g = 0; g < pl.pairs; ++g) load[g] = base_load[g];
   pl.makespan = 0;
   for (int g = 0; g < pl.pairs; ++g)
     if (load[g] > pl.makespan) pl.makespan = load[g];
@@ -907,7 +974,7 @@ size_t carve_apply(ApplyWorkspace& w, char* base, const Plan& pl, int T, int R) 
   w.Hg = reinterpret_cast<__nv_bfloat16*>(base ? base + off : nullptr);
   if (R > 0) off = up(off + (size_t)T * R * sizeof(__nv_bfloat16));
   w.partial = reinterpret_cast<float*>(base ? base + off : nullptr);
-  if (R > 0 && pl.shrink_splits > 1) off = up(off + (size_t)pl.shrink_splits * T * R * sizeof(float));
+  if (R > 0 && pl.shrink_splits > 1) off = up(off + (size_t)pl.shrink_splits * pl.n_m_pairs * 2 * BM * R * sizeof(float));
   w.sk_partial = reinterpret_cast<float*>(base ? base + off : nullptr);
   const bool split = pl.split_k > 1;
   const size_t n_tiles = (size_t)pl.n_m_pairs * pl.n_wide;              // split plans have one tile width
@@ -951,7 +1018,8 @@ cwl_status apply_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, co
     return CWL_ERR_WORKSPACE;
   }
 
-  CUtensorMap mX, mW, mA, mH, mB;
+  CUtensorMap mX, mW, mA, mH, mB, mY;
+  if (!make_map(&mY, Y, (uint64_t)d_out, (uint64_t)T, (uint64_t)ldy, 64, 32)) return CWL_ERR_CUDA;
   if (!make_map(&mX, X, (uint64_t)d_in, (uint64_t)T, (uint64_t)ldx, BK, BM)) return CWL_ERR_CUDA;
   if (!make_map(&mW, W, (uint64_t)d_out, (uint64_t)d_in, (uint64_t)ldw, kBoxCols, BK)) return CWL_ERR_CUDA;
   if (adapter) {
@@ -981,7 +1049,7 @@ cwl_status apply_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, co
     CWL_CUDA_TRY(cudaFuncSetAttribute(apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout::kTotal));
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
-  apply_kernel<<<2 * pl.pairs, kThreads, SmemLayout::kTotal, stream>>>(mX, mW, mA, mH, mB, p);
+  apply_kernel<<<2 * pl.pairs, kThreads, SmemLayout::kTotal, stream>>>(mX, mW, mA, mH, mB, mY, p);
   CWL_CUDA_TRY(cudaGetLastError());
   return CWL_OK;
 }
