@@ -528,6 +528,10 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     uint32_t local = 0;
     Item item;
     for (int i = 0; get_item(i, pair, sh_begin, p, item); ++i, ++local) {
+      if (item.kind == ITEM_SHRINK && epi_tid < BM) {
+        // the row gates of this item's row tile, looked up while the main loop runs (a chain of dependent loads)
+        gates[epi_tid] = row_gate((item.m_pair * 2 + (int)rank) * BM + epi_tid, p);
+      }
       mbar_wait(acc_full_bar, local & 1u, abort_flag);    // a failure is recorded in abort_flag
       // one thread decides for all 256 so that the barriers below are never split
       epilogue_barrier();
@@ -579,23 +583,32 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       }
 
       if (item.kind == ITEM_PROJECT) {
-        // ---- split-K item: store the fp32 partial, then reduce this item's share of the tile's columns ----
-        // partial layout [column group of 4][128 rows][4]: a warp's store and the reducer's loads are contiguous
-        float* mine = p.sk_partial + ((int64_t)(item.tile * pl.split_k + item.split) * 2 + rank) * (BM * pl.w0);
+        // ---- split-K item: every contributor owns a share of the tile's columns.  It stores the OTHER columns of
+        // its fp32 accumulator (layout [column group of 4][128 rows][4]: a warp's store and the owner's loads are
+        // contiguous), waits until all partials of the tile are in, and adds the others' partials of its own
+        // share to what is still in its tensor memory.  This is the pair's last item, so the accumulator is not
+        // handed back before the end, and the operand ring is free: the bf16 result is staged there row by row
+        // and written to Y with contiguous 16-byte stores.
+        const int share = (((item.wt + pl.split_k - 1) / pl.split_k) + 7) & ~7;
+        const int c_lo = min(item.wt, item.split * share), c_hi = min(item.wt, c_lo + share);
+        const int pitch = share * 2 + 16;            // bytes per staged row
+        float* tile_base = p.sk_partial + ((int64_t)(item.tile * pl.split_k) * 2 + rank) * (BM * pl.w0);
+        const int64_t split_stride = (int64_t)2 * BM * pl.w0;
+        float* mine = tile_base + item.split * split_stride;
 #pragma unroll 1
         for (int cc = chalf; cc < n_chunks; cc += 2) {
+          if (cc * 32 >= c_lo && cc * 32 + 32 <= c_hi) continue;   // wholly mine (warp-uniform)
           uint32_t v[32];
           tmem_ld32(t_row + cc * 32, v);
           tmem_ld_wait();
 #pragma unroll
-          for (int q4 = 0; q4 < 8; ++q4)
-            if (cc * 32 + q4 * 4 < item.wt)
+          for (int q4 = 0; q4 < 8; ++q4) {
+            const int col = cc * 32 + q4 * 4;
+            if (col < item.wt && (col < c_lo || col >= c_hi))
               *reinterpret_cast<uint4*>(mine + ((cc * 8 + q4) * BM + row_in_tile) * 4) =
                   make_uint4(v[q4 * 4 + 0], v[q4 * 4 + 1], v[q4 * 4 + 2], v[q4 * 4 + 3]);
+          }
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(leader_acc_empty);
         __threadfence();                             // this thread's partial, device-wide
         epilogue_barrier();
         int* counter = p.sk_counters + item.tile * 2 + rank;
@@ -606,29 +619,42 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         epilogue_barrier();
         if (*epi_go == 0) break;
         __threadfence();
-        // columns [c_lo, c_hi) of the tile are this item's to reduce (multiples of 8).  This is the pair's last
-        // item and its MMAs have retired, so the operand ring is free: the bf16 result is staged there row by row
-        // and written to Y with contiguous 16-byte stores.
-        const int share = (((item.wt + pl.split_k - 1) / pl.split_k) + 7) & ~7;
-        const int c_lo = min(item.wt, item.split * share), c_hi = min(item.wt, c_lo + share);
-        const int n_cg = (c_hi - c_lo) >> 2;
-        const int pitch = share * 2 + 16;            // bytes per staged row
-        const float* tile_base = p.sk_partial + ((int64_t)(item.tile * pl.split_k) * 2 + rank) * (BM * pl.w0);
-        const int64_t split_stride = (int64_t)2 * BM * pl.w0;
-        for (int idx = epi_tid; idx < BM * n_cg; idx += kEpiThreads) {
-          const int r = idx & (BM - 1), cg = idx >> 7;
-          const float* src = tile_base + ((int64_t)((c_lo >> 2) + cg) * BM + r) * 4;
-          float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
+#pragma unroll 1
+        for (int cc = (c_lo >> 5) + ((((c_lo >> 5) & 1) != chalf) ? 1 : 0); cc * 32 < c_hi; cc += 2) {
+          uint32_t v[32];
+          tmem_ld32(t_row + cc * 32, v);
+          tmem_ld_wait();
+          float acc[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) acc[j] = __uint_as_float(v[j]);
+          const float* src0 = tile_base + ((int64_t)(cc * 8) * BM + row_in_tile) * 4;
+#pragma unroll 2
           for (int s = 0; s < pl.split_k; ++s) {
-            const float4 x = __ldcg(reinterpret_cast<const float4*>(src + s * split_stride));
-            sum.x += x.x; sum.y += x.y; sum.z += x.z; sum.w += x.w;
+            if (s == item.split) continue;
+            const float* src = src0 + s * split_stride;
+#pragma unroll
+            for (int q4 = 0; q4 < 8; ++q4) {
+              const int col = cc * 32 + q4 * 4;
+              if (col >= c_lo && col < c_hi) {
+                const float4 x = __ldcg(reinterpret_cast<const float4*>(src + q4 * BM * 4));
+                acc[q4 * 4 + 0] += x.x; acc[q4 * 4 + 1] += x.y; acc[q4 * 4 + 2] += x.z; acc[q4 * 4 + 3] += x.w;
+              }
+            }
           }
-          uint2 o;
-          o.x = pack_bf16(sum.x, sum.y);
-          o.y = pack_bf16(sum.z, sum.w);
-          *reinterpret_cast<uint2*>(base_ptr + r * pitch + cg * 8) = o;
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4) {
+            const int col = cc * 32 + q4 * 4;
+            if (col >= c_lo && col < c_hi) {
+              uint2 o;
+              o.x = pack_bf16(acc[q4 * 4 + 0], acc[q4 * 4 + 1]);
+              o.y = pack_bf16(acc[q4 * 4 + 2], acc[q4 * 4 + 3]);
+              *reinterpret_cast<uint2*>(base_ptr + row_in_tile * pitch + (col - c_lo) * 2) = o;
+            }
+          }
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(leader_acc_empty);
         epilogue_barrier();
         const int pieces = (c_hi - c_lo) >> 3;       // 16-byte pieces per row
         for (int idx = epi_tid; idx < BM * pieces; idx += kEpiThreads) {
@@ -643,8 +669,7 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
 
       // ---- shrink item ----
       const bool direct = pl.shrink_splits == 1;     // no partials: gate straight from the accumulator
-      RowGate g{0.f, 0.f, 0, 0};
-      if (direct) g = row_gate(row, p);
+      const RowGate g = gates[row_in_tile];          // written before the barriers above
 #pragma unroll 1
       for (int cc = chalf; cc < n_chunks; cc += 2) {
         const int col = cc * 32;
@@ -692,8 +717,6 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       if (*epi_last == 0) continue;
       // this CTA completed its row tile: sum the partials, gate, publish H'
       __threadfence();
-      if (epi_tid < BM) gates[epi_tid] = row_gate(m_tile * BM + epi_tid, p);
-      epilogue_barrier();
       const int quads = p.R >> 2;                    // float4 groups per row
       const int64_t split_stride = (int64_t)2 * pl.n_m_pairs * p.R * BM;
       for (int idx = epi_tid; idx < BM * quads; idx += kEpiThreads) {
@@ -794,7 +817,8 @@ Plan make_plan(int T, int d_in, int d_out, int R, int pairs, bool allow_split_k)
       }
       int split_k = 1, kb_per_ksplit = pl.nkb0;
       if (allow_split_k && n_narrow == 0 && 2 * NW <= pairs) {
-        const int spare = R > 0 ? (pairs >= 16 ? pairs / 9 : 0) : 0;    // pairs left free for the shrink items
+        const int spare = pairs >= 16 ? pairs / 9 : 0;   // pairs left free for shrink items (also without an adapter,
+                                                         // so that the plan and its workspace do not depend on R)
         int s = (pairs - spare) / NW;
         const int min_kb = 8;                                           // K blocks per item, at least
         if (s > pl.nkb0 / min_kb) s = pl.nkb0 / min_kb;
