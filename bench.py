@@ -43,13 +43,23 @@ def load_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
-def load_traffic(kernel: str):
-    """DRAM bytes per launch of the dominant kernel from a committed ncu summary, or None."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
+# Revision tag of the dominant kernel the ncu counters under profiles/ were taken on.  Bump it whenever
+# cwl_apply's kernel changes: a traffic figure taken on another revision is reported as null.
+APPLY_KERNEL_REVISION = "pairs-256x512-planned-tma-store"
+
+
+def load_traffic(key: str):
+    """DRAM bytes per step of the dominant kernel from the committed ncu summary, or None when there is
+    no figure for this workload or the kernel has changed since the counters were taken."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
     if not os.path.exists(path):
         return None
     with open(path) as fh:
-        return json.load(fh).get(kernel)
+        for line in fh:
+            parts = line.split()
+            if len(parts) >= 3 and not line.startswith("#") and parts[0] == key and parts[2] == APPLY_KERNEL_REVISION:
+                return float(parts[1])
+    return None
 
 
 class ClockSampler:
@@ -353,7 +363,8 @@ def run_ours(args):
         roof = {"bound": "tensor", "achieved": achieved, "peak": peaks[kind], "unit": "TFLOP/s",
                 "frac": achieved / peaks[kind], "traffic": load_traffic("apply_" + args.workload),
                 "peak_source": f"{kind}, of {peaks['source']}"}
-    roof["kernel"] = "cwl_apply (shrink + gate + projection GEMM; the event bracket spans all launches of the 7 applies of a step)"
+    roof["kernel"] = ("cwl::apply_kernel (one fused launch per projection: shrink, gate, base GEMM + expand); achieved = the "
+                      "step's algorithmic FLOPs or bytes over the event-timed span of its apply launches")
     roof["launch_ms"] = apply_avg_ms
     roof["executed_tflops"] = f_exe / (apply_avg_ms * 1e-3) / 1e12
     roof["frac_of_nominal_2250"] = (f_alg / (apply_avg_ms * 1e-3) / 1e12) / 2250.0
