@@ -781,8 +781,9 @@ int shrink_splits_for(int T, int d_in) {
 }
 
 // Chooses tile widths, the K split and who does the shrink work for `pairs` resident CTA pairs.
-// Depends on the shape and on `pairs` only.  allow_split_k = false keeps every tile whole.
-Plan make_plan(int T, int d_in, int d_out, int R, int pairs, bool allow_split_k) {
+// Depends on the shape and on `pairs` only.  allow_split_k = false keeps every tile whole; scratch_limit > 0
+// keeps the shrink's split small enough for H' and the partial sums to fit that many bytes (one split always may).
+Plan make_plan(int T, int d_in, int d_out, int R, int pairs, bool allow_split_k, size_t scratch_limit = 0) {
   Plan pl;
   memset(&pl, 0, sizeof(pl));
   if (pairs > kPairsPlanned) pairs = kPairsPlanned;
@@ -869,6 +870,8 @@ Plan make_plan(int T, int d_in, int d_out, int R, int pairs, bool allow_split_k)
     for (int want = 1; want <= kMaxSplits; want *= 2) {
       if (want > pl.nkb0) break;
       const int per = ceil_div(pl.nkb0, want), splits = ceil_div(pl.nkb0, per);
+      const size_t scratch = (size_t)T * R * 2 + (size_t)splits * pl.n_m_pairs * 2 * BM * R * 4 + 4096 + 16 * (size_t)pl.n_m_pairs;
+      if (scratch_limit > 0 && splits > 1 && scratch > scratch_limit) continue;
       const long long cs = (long long)per * (16 + 8 * boxes_for(R / 2)) + 176;
       const int n_shrink = pl.n_m_pairs * splits;
       uint16_t count[kPairsPlanned];
@@ -1013,7 +1016,8 @@ size_t carve_apply(ApplyWorkspace& w, char* base, const Plan& pl, int T, int R) 
 cwl_status apply_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, const void* A, int64_t lda,
                       const void* B, int64_t ldb, int32_t T, int32_t d_in, int32_t d_out, int32_t R,
                       cwl_chunk_table table, int32_t window, void* Y, int64_t ldy, void* workspace,
-                      size_t workspace_bytes, int32_t* status_word, void* stream_, bool allow_split_k) {
+                      size_t workspace_bytes, int32_t* status_word, void* stream_, bool allow_split_k,
+                      size_t scratch_limit = 0) {
   if (T < 0 || d_in < 1 || d_out < 1 || R < 0 || window < 0) return CWL_ERR_INVALID_ARG;
   if (T > 0 && (X == nullptr || Y == nullptr)) return CWL_ERR_INVALID_ARG;
   if (W == nullptr) return CWL_ERR_INVALID_ARG;
@@ -1032,12 +1036,12 @@ cwl_status apply_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, co
   const int Reff = adapter ? R : 0;
 
   ApplyWorkspace ws{nullptr, nullptr, nullptr, nullptr, 0};
-  Plan pl = make_plan(T, d_in, d_out, Reff, max_pairs(), allow_split_k);
+  Plan pl = make_plan(T, d_in, d_out, Reff, max_pairs(), allow_split_k, scratch_limit);
   const size_t need = carve_apply(ws, static_cast<char*>(workspace), pl, T, Reff);
   const bool have_ws = workspace != nullptr && workspace_bytes >= need && (reinterpret_cast<uintptr_t>(workspace) & 255u) == 0;
   if (!have_ws && !adapter && pl.split_k > 1) {
     // the plain projection needs scratch only when its K loop is split; without a workspace it runs unsplit
-    pl = make_plan(T, d_in, d_out, Reff, max_pairs(), false);
+    pl = make_plan(T, d_in, d_out, Reff, max_pairs(), false, scratch_limit);
   } else if (!have_ws && (adapter || pl.split_k > 1)) {
     return CWL_ERR_WORKSPACE;
   }
@@ -1150,7 +1154,7 @@ cwl_status noalloc_scratch(void** out) {
 extern "C" size_t cwl_apply_noalloc_scratch_need(int32_t T, int32_t d_in, int32_t d_out, int32_t R) {
   if (T <= 0 || d_in <= 0 || d_out <= 0 || R < 0) return 256;
   cwl::ApplyWorkspace w;
-  const cwl::Plan pl = cwl::make_plan(T, d_in, d_out, R, cwl::max_pairs(), false);
+  const cwl::Plan pl = cwl::make_plan(T, d_in, d_out, R, cwl::max_pairs(), false, CWL_NOALLOC_SCRATCH_BYTES);
   return cwl::carve_apply(w, nullptr, pl, T, R);
 }
 
@@ -1168,5 +1172,5 @@ extern "C" cwl_status cwl_apply_noalloc(const void* X, int64_t ldx, const void* 
   if (st != CWL_OK) return st;
   // every tile keeps its whole K loop here: the partial accumulators of a split K loop would not fit
   return cwl::apply_impl(X, ldx, W, ldw, A, lda, B, ldb, T, d_in, d_out, R, table, window, Y, ldy, scratch,
-                         (size_t)CWL_NOALLOC_SCRATCH_BYTES, status_word, stream, false);
+                         (size_t)CWL_NOALLOC_SCRATCH_BYTES, status_word, stream, false, CWL_NOALLOC_SCRATCH_BYTES);
 }

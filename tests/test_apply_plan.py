@@ -70,3 +70,6 @@ def test_plan_rejects_bad_shapes():
 def test_workspace_grows_with_the_split_and_noalloc_need_does_not():
     assert cwl.cwl_apply_workspace_bytes(256, 4096, 11008, 64) > cwl.cwl_apply_noalloc_scratch_need(256, 4096, 11008, 64)
     assert cwl.cwl_apply_noalloc_scratch_need(2048, 4096, 4096, 64) <= cwl.NOALLOC_SCRATCH_BYTES
+    for T in (8192, 16384, 32768):                       # the documented reach of the built-in scratch at R = 64
+        assert cwl.cwl_apply_noalloc_scratch_need(T, 4096, 11008, 64) <= cwl.NOALLOC_SCRATCH_BYTES
+    assert cwl.cwl_apply_noalloc_scratch_need(65536, 4096, 4096, 64) > cwl.NOALLOC_SCRATCH_BYTES
