@@ -35,7 +35,7 @@ def policy_struct(p: Policy) -> cwl.CPolicy:
 class HotPath:
     """Device-resident state of one layer's adapted projections plus the scheduler in front."""
 
-    def __init__(self, w: Workload, device: str = "cuda", keep_host: bool = False):
+    def __init__(self, w: Workload, device: str = "cuda", keep_host: bool = False, n_layers: int = 1):
         self.T, self.R, self.policy = w.T, w.R, w.policy
         self.device = device
         self.cu_seqlens = torch.from_numpy(w.cu_seqlens).to(device)
@@ -49,6 +49,13 @@ class HotPath:
             self.projs.append(DeviceProjection(
                 p.name, p.d_in, p.d_out, cwl.bf16_from_bits(p.W, device), cwl.bf16_from_bits(p.A, device),
                 cwl.bf16_from_bits(p.B, device), torch.empty(w.T, p.d_out, dtype=torch.bfloat16, device=device)))
+        # a stack of layers: every layer has its own weights and adapter factors in HBM (distinct memory, so a
+        # layer never finds its weights in L2); layers beyond the first hold the first layer's values rolled by
+        # one row per layer, which is all a timing run needs
+        self.layers: List[List[DeviceProjection]] = [self.projs]
+        for l in range(1, n_layers):
+            self.layers.append([DeviceProjection(p.name, p.d_in, p.d_out, torch.roll(p.W, l, 0), torch.roll(p.A, l, 0),
+                                                 torch.roll(p.B, l, 1), p.Y) for p in self.projs])
         cap = w.T // max(w.policy.min_len, 1) + self.n_seq + 1
         self.table = cwl.DeviceChunkTable(cap, device)
         if w.table is not None:
@@ -78,19 +85,20 @@ class HotPath:
         cwl.cwl_partition(self.score, self.cu_seqlens, self.cpolicy, table=self.table, workspace=self.part_ws,
                           status_word=self.status)
 
-    def apply_step(self, table: Optional[cwl.DeviceChunkTable] = None, dense: bool = False) -> None:
+    def apply_step(self, table: Optional[cwl.DeviceChunkTable] = None, dense: bool = False, layer: int = 0) -> None:
         tab = table if table is not None else self.table
-        for p in self.projs:
+        for p in self.layers[layer]:
             cwl.cwl_apply(self.X[p.d_in], p.W, None if dense else p.A, None if dense else p.B, tab,
                           self.policy.window, Y=p.Y, workspace=self.apply_ws, status_word=self.status)
 
     def step(self) -> None:
         """One pass of the whole hot path on the current stream (no host synchronisation)."""
-        if self.logits is not None:
-            self.score_step()
-        if not self.fixed_table:
-            self.partition_step()
-        self.apply_step()
+        for layer in range(len(self.layers)):
+            if self.logits is not None:
+                self.score_step()
+            if not self.fixed_table:
+                self.partition_step()
+            self.apply_step(layer=layer)
 
     def launches_per_step(self) -> int:
         n = self.LAUNCHES_APPLY * len(self.projs)
@@ -98,4 +106,4 @@ class HotPath:
             n += self.LAUNCHES_SCORE
         if not self.fixed_table:
             n += self.LAUNCHES_PARTITION
-        return n
+        return n * len(self.layers)
