@@ -125,6 +125,30 @@ cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64_t ldw,
                      void* workspace, size_t workspace_bytes,
                      int32_t* status_word, void* stream);
 
+/* Several adapted projections of the SAME rows in one launch (Sec. III-F: the adapter sits on every attention and
+ * MLP projection; q, k, v read one activation, gate and up another).  Projection j computes
+ *   Y_j = X W_j + gated (X A_j) B_j
+ * exactly as cwl_apply does, with the chunk table, window, d_in and R shared by the group.  One pass over X serves
+ * all shrinks, and the output tiles of all projections are scheduled together, which fills the last wave of tiles
+ * better than separate calls.  Meant for prefill-sized T; decode-sized T is better served by separate cwl_apply
+ * calls, whose K loop is split.
+ *   proj        HOST array of n_proj descriptors (1 <= n_proj <= CWL_MAX_GROUP), copied at call time; all pointers
+ *               inside are DEV.  Either every projection has A and B, or none has.
+ *   workspace   DEV, at least cwl_apply_grouped_workspace_bytes(T, d_in, n_proj, d_out[], R) bytes, 256-byte aligned
+ * Shape rules and errors as for cwl_apply, plus UNSUPPORTED when n_proj * R > 512. */
+#define CWL_MAX_GROUP 4
+typedef struct {
+  const void* W; int64_t ldw;   /* DEV bf16 [d_in, d_out] */
+  const void* A; int64_t lda;   /* DEV bf16 [d_in, R] or NULL */
+  const void* B; int64_t ldb;   /* DEV bf16 [R, d_out] or NULL */
+  void*       Y; int64_t ldy;   /* DEV bf16 [T, d_out] */
+  int32_t d_out;
+} cwl_projection;
+size_t     cwl_apply_grouped_workspace_bytes(int32_t T, int32_t d_in, int32_t n_proj, const int32_t* d_out, int32_t R);
+cwl_status cwl_apply_grouped(const void* X, int64_t ldx, const cwl_projection* proj, int32_t n_proj,
+                             int32_t T, int32_t d_in, int32_t R, cwl_chunk_table table, int32_t window,
+                             void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream);
+
 /* The schedule cwl_apply uses for a shape when `pairs` CTA pairs can be resident (a B200 holds 74): how
  * the output is cut into column tiles (Sec. III-F leaves the kernel schedule open; this is the library's own
  * design), whether the K loop of decode-sized problems is split, and who computes the shrink X A.

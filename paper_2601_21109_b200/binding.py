@@ -20,7 +20,8 @@ STATUS = {0: "CWL_OK", 1: "CWL_ERR_INVALID_ARG", 2: "CWL_ERR_SHAPE", 3: "CWL_ERR
           4: "CWL_ERR_CAPACITY", 5: "CWL_ERR_WORKSPACE", 6: "CWL_ERR_CUDA", 7: "CWL_ERR_TIMEOUT"}
 
 EXPORTS = ["cwl_status_string", "cwl_version", "cwl_score_tokens", "cwl_partition_workspace_bytes",
-           "cwl_partition", "cwl_apply_workspace_bytes", "cwl_apply", "cwl_apply_plan",
+           "cwl_partition", "cwl_apply_workspace_bytes", "cwl_apply", "cwl_apply_grouped_workspace_bytes",
+           "cwl_apply_grouped", "cwl_apply_plan",
            "cwl_apply_noalloc_scratch_need", "cwl_apply_noalloc"]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 
@@ -44,6 +45,14 @@ class CChunkTable(C.Structure):
     _fields_ = [("offsets", C.c_void_p), ("rank", C.c_void_p), ("scale", C.c_void_p),
                 ("rung", C.c_void_p), ("flags", C.c_void_p), ("n_chunks", C.c_void_p),
                 ("capacity", C.c_int32)]
+
+
+MAX_GROUP = 4
+
+
+class CProjection(C.Structure):
+    _fields_ = [("W", C.c_void_p), ("ldw", C.c_int64), ("A", C.c_void_p), ("lda", C.c_int64),
+                ("B", C.c_void_p), ("ldb", C.c_int64), ("Y", C.c_void_p), ("ldy", C.c_int64), ("d_out", C.c_int32)]
 
 
 class CApplyPlanInfo(C.Structure):
@@ -81,6 +90,11 @@ def lib():
                                 C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                 CChunkTable, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t,
                                 C.c_void_p, C.c_void_p]
+        L.cwl_apply_grouped_workspace_bytes.restype = C.c_size_t
+        L.cwl_apply_grouped_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_int32), C.c_int32]
+        L.cwl_apply_grouped.restype = C.c_int
+        L.cwl_apply_grouped.argtypes = [C.c_void_p, C.c_int64, C.POINTER(CProjection), C.c_int32, C.c_int32, C.c_int32,
+                                        C.c_int32, CChunkTable, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         L.cwl_apply_plan.restype = C.c_int
         L.cwl_apply_plan.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(CApplyPlanInfo)]
         L.cwl_apply_noalloc_scratch_need.restype = C.c_size_t
@@ -232,6 +246,37 @@ def cwl_apply(X: torch.Tensor, W: torch.Tensor, A: Optional[torch.Tensor], B: Op
                                         T, d_in, d_out, R, ct, int(window), _p(Y), Y.stride(0),
                                         _p(workspace), workspace.numel(), _p(status_word), _stream_ptr(stream)))
     return Y
+
+
+def cwl_apply_grouped_workspace_bytes(T: int, d_in: int, d_outs: Sequence[int], R: int) -> int:
+    arr = (C.c_int32 * len(d_outs))(*[int(d) for d in d_outs])
+    return int(lib().cwl_apply_grouped_workspace_bytes(T, d_in, len(d_outs), arr, R))
+
+
+def cwl_apply_grouped(X: torch.Tensor, Ws: Sequence[torch.Tensor], As: Optional[Sequence[torch.Tensor]],
+                      Bs: Optional[Sequence[torch.Tensor]], table: Optional[DeviceChunkTable], window: int,
+                      Ys: Optional[Sequence[torch.Tensor]] = None, workspace: Optional[torch.Tensor] = None,
+                      status_word: Optional[torch.Tensor] = None,
+                      stream: Optional[torch.cuda.Stream] = None) -> Sequence[torch.Tensor]:
+    """Y_j = X W_j + gated (X A_j) B_j for up to four projections of the same rows, one launch."""
+    T, d_in = X.shape
+    n = len(Ws)
+    R = As[0].shape[1] if (As is not None and Bs is not None) else 0
+    if Ys is None:
+        Ys = [torch.empty(T, W.shape[1], dtype=torch.bfloat16, device=X.device) for W in Ws]
+    if workspace is None:
+        workspace = torch.empty(cwl_apply_grouped_workspace_bytes(T, d_in, [W.shape[1] for W in Ws], R),
+                                dtype=torch.uint8, device=X.device)
+    arr = (CProjection * n)()
+    for j in range(n):
+        arr[j] = CProjection(_p(Ws[j]), Ws[j].stride(0), _p(As[j]) if R else None, As[j].stride(0) if R else 0,
+                             _p(Bs[j]) if R else None, Bs[j].stride(0) if R else 0, _p(Ys[j]), Ys[j].stride(0),
+                             Ws[j].shape[1])
+    ct = table.c_struct() if table is not None else CChunkTable(None, None, None, None, None, None, 0)
+    _check("cwl_apply_grouped", lib().cwl_apply_grouped(_p(X), X.stride(0), arr, n, T, d_in, R, ct, int(window),
+                                                        _p(workspace), workspace.numel(), _p(status_word),
+                                                        _stream_ptr(stream)))
+    return Ys
 
 
 def cwl_apply_noalloc(X: torch.Tensor, W: torch.Tensor, A: Optional[torch.Tensor], B: Optional[torch.Tensor],

@@ -74,8 +74,12 @@ struct Plan {
   int pairs;                  // CTA pairs launched
   int n_m_pairs;              // 256-row tiles
   int nkb0, nkb1;             // K blocks over d_in, over R
-  int w0, n_wide;             // wide column tiles per pair row: columns [0, n_wide * w0)
-  int w1, n_narrow;           // then n_narrow tiles of width w1 (the last one may be ragged)
+  int n_proj;                 // projections sharing X and the chunk table (1 for cwl_apply)
+  int d_out[CWL_MAX_GROUP];   // their output widths
+  int w0, n_wide;             // wide column tiles per pair row, all projections together
+  int w1, n_narrow;           // narrow tiles per pair row, all projections together
+  int pw[CWL_MAX_GROUP];      // projection j: columns [0, pw[j] * w0) in wide tiles,
+  int pn[CWL_MAX_GROUP];      //               then pn[j] tiles of width w1 (the last tile of a projection may be ragged)
   int split_k, kb_per_ksplit; // split of the d_in blocks of every tile (1 = none); only when all items fit one wave
   int shrink_splits, kb_per_split;
   int boxes;                  // right-operand boxes per CTA per stage, at most
@@ -85,11 +89,12 @@ struct Plan {
 };
 
 struct ApplyParams {
-  int T, d_in, d_out, R;   // R = 0: no adapter
+  int T, d_in, R;          // R = 0: no adapter
+  int RT;                  // n_proj * R: columns of the shrink output, all projections side by side
   int window;
-  __nv_bfloat16* Y; int64_t ldy;
-  __nv_bfloat16* Hg;       // [T, R] gated shrink output
-  float* partial;          // [shrink_splits, 128-row tiles, R / 4, 128, 4] fp32 partial shrink sums
+  __nv_bfloat16* Y[CWL_MAX_GROUP]; int64_t ldy[CWL_MAX_GROUP];
+  __nv_bfloat16* Hg;       // [T, RT] gated shrink outputs
+  float* partial;          // [shrink_splits, 128-row tiles, RT / 4, 128, 4] fp32 partial shrink sums
   float* sk_partial;       // [tiles * split_k * 2, 128, w0] fp32 partial accumulators of split-K items
   int* counters;           // [2 n_m_pairs] shrink splits finished per 128-row tile
   int* flags;              // [2 n_m_pairs] 1 once H' of the 128-row tile is published
@@ -97,6 +102,12 @@ struct ApplyParams {
   cwl_chunk_table table;
   int32_t* status_word;
   Plan plan;
+};
+
+// Tensor maps of one launch: X and H' are shared, the rest is per projection.
+struct GroupMaps {
+  CUtensorMap x, h;
+  CUtensorMap w[CWL_MAX_GROUP], a[CWL_MAX_GROUP], b[CWL_MAX_GROUP], y[CWL_MAX_GROUP];
 };
 
 // ------------------------------------------------------------------------------------------ PTX
@@ -258,6 +269,7 @@ __host__ __device__ __forceinline__ int boxes_for(int cols_per_cta) { return (co
 enum : int { ITEM_SHRINK = 0, ITEM_PROJECT = 1 };
 struct Item {
   int kind, m_pair;
+  int proj;             // project: which projection of the group
   int n0, wt;           // first column and width (multiple of 16) of the tile; shrink: 0, R
   int split;            // shrink: which split of d_in.  project: which K split
   int tile;             // project: index of the output tile (for split-K bookkeeping)
@@ -289,7 +301,7 @@ __device__ __forceinline__ bool get_item(int i, int b, int sh_begin, const Apply
   if (i < my_shrink) {
     const int s = sh_begin + i;
     it.kind = ITEM_SHRINK; it.m_pair = s / pl.shrink_splits; it.split = s - it.m_pair * pl.shrink_splits;
-    it.n0 = 0; it.wt = p.R; it.tile = 0;
+    it.n0 = 0; it.wt = p.RT; it.tile = 0; it.proj = 0;
     it.kb0 = it.split * pl.kb_per_split;
     it.n_blk0 = min(pl.nkb0, it.kb0 + pl.kb_per_split) - it.kb0;
     it.n_blk1 = 0;
@@ -301,16 +313,18 @@ __device__ __forceinline__ bool get_item(int i, int b, int sh_begin, const Apply
   const int n_tiles = n_wide_tiles + n_narrow_tiles;
   if (idx >= n_tiles * pl.split_k) return false;
   const int tile = idx / pl.split_k, ks = idx - tile * pl.split_k;
-  int c, w;
+  int c, w, j = 0;
   if (tile < n_wide_tiles) {
     raster(tile, pl.n_m_pairs, pl.n_wide, it.m_pair, c);
+    while (c >= pl.pw[j]) { c -= pl.pw[j]; ++j; }
     it.n0 = c * pl.w0; w = pl.w0;
   } else {
     raster(tile - n_wide_tiles, pl.n_m_pairs, pl.n_narrow, it.m_pair, c);
-    it.n0 = pl.n_wide * pl.w0 + c * pl.w1; w = pl.w1;
+    while (c >= pl.pn[j]) { c -= pl.pn[j]; ++j; }
+    it.n0 = pl.pw[j] * pl.w0 + c * pl.w1; w = pl.w1;
   }
-  it.kind = ITEM_PROJECT; it.tile = tile; it.split = ks;
-  it.wt = min(w, p.d_out - it.n0);             // d_out and the widths are multiples of 16
+  it.kind = ITEM_PROJECT; it.tile = tile; it.split = ks; it.proj = j;
+  it.wt = min(w, pl.d_out[j] - it.n0);         // d_out and the widths are multiples of 16
   it.kb0 = ks * pl.kb_per_ksplit;
   it.n_blk0 = min(pl.nkb0, it.kb0 + pl.kb_per_ksplit) - it.kb0;
   it.n_blk1 = (ks == pl.split_k - 1) ? pl.nkb1 : 0;
@@ -369,10 +383,7 @@ static_assert(BM * sizeof(RowGate) <= SmemLayout::kOutBytes, "row gates must fit
 static_assert(SmemLayout::kTotal <= 227 * 1024, "shared memory budget");
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
-             const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_h,
-             const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_y,
-             const __grid_constant__ ApplyParams p) {
+apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ ApplyParams p) {
   using L = SmemLayout;
   constexpr uint32_t kTmemCols = kMaxTileW;
 
@@ -409,10 +420,13 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     mbar_init(acc_empty_bar, 2 * kEpiWarps);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    prefetch_tmap(&tm_x);
-    prefetch_tmap(&tm_w);
-    prefetch_tmap(&tm_y);
-    if (p.R > 0) { prefetch_tmap(&tm_a); prefetch_tmap(&tm_h); prefetch_tmap(&tm_b); }
+    prefetch_tmap(&tm.x);
+    for (int j = 0; j < p.plan.n_proj; ++j) {
+      prefetch_tmap(&tm.w[j]);
+      prefetch_tmap(&tm.y[j]);
+      if (p.R > 0) { prefetch_tmap(&tm.a[j]); prefetch_tmap(&tm.b[j]); }
+    }
+    if (p.R > 0) prefetch_tmap(&tm.h);
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
@@ -436,12 +450,14 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       for (int i = 0; ok && get_item(i, pair, sh_begin, p, item); ++i) {
         const bool shrink = item.kind == ITEM_SHRINK;
         const int m_tile = item.m_pair * 2 + (int)rank;       // this CTA's 128-row tile
-        // columns of the right operand this CTA supplies: its half of each MMA's columns
-        const int ca = item.wa >> 1, cb = item.wb >> 1;
+        // columns of the right operand this CTA supplies: its half of each MMA's columns.  A shrink item runs
+        // one MMA of N = R per projection (their A factors are separate matrices); a projection tile runs one or two.
+        const int ca = shrink ? (p.R >> 1) : (item.wa >> 1), cb = shrink ? 0 : (item.wb >> 1);
         const int boxes_a = boxes_for(ca), boxes_b = boxes_for(cb);
-        const int col_a = item.n0 + (int)rank * ca, col_b = item.n0 + item.wa + (int)rank * cb;
-        const uint32_t tx_pair = 2u * (kABytes + (boxes_a + boxes_b) * kBoxBytes);
-        const CUtensorMap* right0 = shrink ? &tm_a : &tm_w;
+        const int col_a = shrink ? (int)rank * ca : item.n0 + (int)rank * ca;
+        const int col_b = item.n0 + item.wa + (int)rank * cb;
+        const int n_right = shrink ? pl.n_proj : 1;           // matrices the first group of boxes comes from
+        const uint32_t tx_pair = 2u * (kABytes + (n_right * boxes_a + boxes_b) * kBoxBytes);
         const int n_blk = item.n_blk0 + item.n_blk1;
         for (int b = 0; b < n_blk; ++b, ++it_cnt) {
           const int s = it_cnt % n_stages;
@@ -454,14 +470,17 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             fence_proxy_async();
           }
           const int k = phase1 ? (b - item.n_blk0) * BK : (item.kb0 + b) * BK;
-          const CUtensorMap* left = phase1 ? &tm_h : &tm_x;
-          const CUtensorMap* right = phase1 ? &tm_b : right0;
           const uint32_t sa = base + s * stage_bytes, sb = sa + kABytes;
           const uint32_t leader_full = mapa_shared(full_bar(s), 0); // the same barrier in the leader's shared memory
           if (rank == 0) mbar_expect_tx(full_bar(s), tx_pair);
-          tma_load_2d_pair(sa, left, leader_full, k, m_tile * BM);
-          for (int j = 0; j < boxes_a; ++j)
-            tma_load_2d_pair(sb + j * kBoxBytes, right, leader_full, col_a + j * kBoxCols, k);
+          if (phase1) tma_load_2d_pair(sa, &tm.h, leader_full, item.proj * p.R + k, m_tile * BM);
+          else tma_load_2d_pair(sa, &tm.x, leader_full, k, m_tile * BM);
+          for (int q = 0; q < n_right; ++q) {
+            const CUtensorMap* right = shrink ? &tm.a[q] : (phase1 ? &tm.b[item.proj] : &tm.w[item.proj]);
+            for (int j = 0; j < boxes_a; ++j)
+              tma_load_2d_pair(sb + (q * boxes_a + j) * kBoxBytes, right, leader_full, col_a + j * kBoxCols, k);
+          }
+          const CUtensorMap* right = phase1 ? &tm.b[item.proj] : &tm.w[item.proj];
           for (int j = 0; j < boxes_b; ++j)
             tma_load_2d_pair(sb + (boxes_a + j) * kBoxBytes, right, leader_full, col_b + j * kBoxCols, k);
         }
@@ -482,9 +501,11 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       bool ok = true;
       Item item;
       for (int i = 0; ok && get_item(i, pair, sh_begin, p, item); ++i, ++local) {
-        const uint32_t idesc_a = make_idesc(2 * BM, item.wa);
+        const bool shrink = item.kind == ITEM_SHRINK;
+        const uint32_t idesc_a = make_idesc(2 * BM, shrink ? p.R : item.wa);
         const uint32_t idesc_b = make_idesc(2 * BM, item.wb > 0 ? item.wb : 16);
         const uint32_t sb_off_b = (uint32_t)boxes_for(item.wa >> 1) * kBoxBytes;
+        const uint32_t sb_step_r = (uint32_t)boxes_for(p.R >> 1) * kBoxBytes;   // shrink: boxes of one projection's A
         if (!mbar_wait(acc_empty_bar, (local & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const int n_blk = item.n_blk0 + item.n_blk1;
@@ -503,7 +524,12 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             const uint64_t da = make_smem_desc(sa + kk * (UMMA_K * 2), 16, 1024);
             const uint64_t db = make_smem_desc(sb + kk * (UMMA_K * 128), kBoxBytes, 1024);
             umma_bf16_pair(tmem_base, da, db, idesc_a, acc_flag);
-            if (item.wb > 0) {
+            if (shrink) {
+              for (int q = 1; q < pl.n_proj; ++q) {
+                const uint64_t dq = make_smem_desc(sb + q * sb_step_r + kk * (UMMA_K * 128), kBoxBytes, 1024);
+                umma_bf16_pair(tmem_base + q * p.R, da, dq, idesc_a, acc_flag);
+              }
+            } else if (item.wb > 0) {
               const uint64_t db2 = make_smem_desc(sb + sb_off_b + kk * (UMMA_K * 128), kBoxBytes, 1024);
               umma_bf16_pair(tmem_base + kMmaN, da, db2, idesc_b, acc_flag);
             }
@@ -572,7 +598,7 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
           fence_proxy_async();                       // the staged rows, visible to the TMA engine
           __syncwarp();
           if (lane == 0 && row0 < p.T) {
-            tma_store_2d(&tm_y, obuf, item.n0 + c64 * 64, row0);
+            tma_store_2d(&tm.y[item.proj], obuf, item.n0 + c64 * 64, row0);
             bulk_commit();
           }
         }
@@ -662,7 +688,7 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
           const int t = m_tile * BM + r;
           if (t >= p.T) break;
           const uint4 q = *reinterpret_cast<const uint4*>(base_ptr + r * pitch + pc * 16);
-          *reinterpret_cast<uint4*>(p.Y + (int64_t)t * p.ldy + item.n0 + c_lo + pc * 8) = q;
+          *reinterpret_cast<uint4*>(p.Y[item.proj] + (int64_t)t * p.ldy[item.proj] + item.n0 + c_lo + pc * 8) = q;
         }
         continue;
       }
@@ -678,19 +704,19 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         tmem_ld_wait();
         if (!direct) {
           // partial layout [split][128-row tile][column group of 4][128 rows][4]: contiguous per warp store
-          float* out = p.partial + (((int64_t)(item.split * 2 * pl.n_m_pairs + m_tile) * (p.R >> 2) + cc * 8) * BM + row_in_tile) * 4;
+          float* out = p.partial + (((int64_t)(item.split * 2 * pl.n_m_pairs + m_tile) * (p.RT >> 2) + cc * 8) * BM + row_in_tile) * 4;
 #pragma unroll
           for (int q4 = 0; q4 < 8; ++q4) {
-            if (col + q4 * 4 < p.R)
+            if (col + q4 * 4 < p.RT)
               *reinterpret_cast<uint4*>(out + q4 * BM * 4) = make_uint4(v[q4 * 4 + 0], v[q4 * 4 + 1], v[q4 * 4 + 2], v[q4 * 4 + 3]);
           }
         } else if (row < p.T) {
           {
-            __nv_bfloat16* out = p.Hg + (int64_t)row * p.R + col;
+            __nv_bfloat16* out = p.Hg + (int64_t)row * p.RT + col;
 #pragma unroll
             for (int q8 = 0; q8 < 4; ++q8) {
-              if (col + q8 * 8 < p.R) {
-                const int j = col + q8 * 8;
+              if (col + q8 * 8 < p.RT) {
+                const int j = (col + q8 * 8) % p.R;      // rank index inside its projection (R is a multiple of 8)
                 uint4 q;
                 q.x = pack_bf16(__uint_as_float(v[q8 * 8 + 0]) * gate_at(g, j + 0), __uint_as_float(v[q8 * 8 + 1]) * gate_at(g, j + 1));
                 q.y = pack_bf16(__uint_as_float(v[q8 * 8 + 2]) * gate_at(g, j + 2), __uint_as_float(v[q8 * 8 + 3]) * gate_at(g, j + 3));
@@ -717,10 +743,10 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       if (*epi_last == 0) continue;
       // this CTA completed its row tile: sum the partials, gate, publish H'
       __threadfence();
-      const int quads = p.R >> 2;                    // float4 groups per row
-      const int64_t split_stride = (int64_t)2 * pl.n_m_pairs * p.R * BM;
+      const int quads = p.RT >> 2;                   // float4 groups per row
+      const int64_t split_stride = (int64_t)2 * pl.n_m_pairs * p.RT * BM;
       for (int idx = epi_tid; idx < BM * quads; idx += kEpiThreads) {
-        const int r = idx & (BM - 1), cg = idx >> 7, j0 = cg << 2;
+        const int r = idx & (BM - 1), cg = idx >> 7, jt = cg << 2, j0 = jt % p.R;   // column, rank index in its projection
         const int t = m_tile * BM + r;
         if (t >= p.T) continue;
         const RowGate gr = gates[r];
@@ -734,7 +760,7 @@ apply_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         uint2 o;
         o.x = pack_bf16(sum.x * gate_at(gr, j0), sum.y * gate_at(gr, j0 + 1));
         o.y = pack_bf16(sum.z * gate_at(gr, j0 + 2), sum.w * gate_at(gr, j0 + 3));
-        *reinterpret_cast<uint2*>(p.Hg + (int64_t)t * p.R + j0) = o;
+        *reinterpret_cast<uint2*>(p.Hg + (int64_t)t * p.RT + jt) = o;
       }
       __threadfence();
       epilogue_barrier();
@@ -783,11 +809,19 @@ int shrink_splits_for(int T, int d_in) {
 // Chooses tile widths, the K split and who does the shrink work for `pairs` resident CTA pairs.
 // Depends on the shape and on `pairs` only.  allow_split_k = false keeps every tile whole; scratch_limit > 0
 // keeps the shrink's split small enough for H' and the partial sums to fit that many bytes (one split always may).
-Plan make_plan(int T, int d_in, int d_out, int R, int pairs, bool allow_split_k, size_t scratch_limit = 0) {
+Plan make_plan(int T, int d_in, int n_proj, const int* d_out, int R, int pairs, bool allow_split_k,
+               size_t scratch_limit = 0) {
   Plan pl;
   memset(&pl, 0, sizeof(pl));
   if (pairs > kPairsPlanned) pairs = kPairsPlanned;
   if (pairs < 1) pairs = 1;
+  pl.n_proj = n_proj;
+  int max_dout = 0, max_floor = 0;
+  for (int j = 0; j < n_proj; ++j) {
+    pl.d_out[j] = d_out[j];
+    if (d_out[j] > max_dout) max_dout = d_out[j];
+    if (d_out[j] / kMaxTileW > max_floor) max_floor = d_out[j] / kMaxTileW;
+  }
   pl.n_m_pairs = ceil_div(T, 2 * BM);
   pl.nkb0 = ceil_div(d_in, BK);
   pl.nkb1 = R > 0 ? ceil_div(R, BK) : 0;
@@ -796,19 +830,29 @@ Plan make_plan(int T, int d_in, int d_out, int R, int pairs, bool allow_split_k,
   pl.kb_per_split = ceil_div(pl.nkb0, pl.shrink_splits);
   pl.split_k = 1; pl.kb_per_ksplit = pl.nkb0;
 
-  // ---- column tiling: n_wide tiles of 512 and the rest in tiles of w1, or (decode-sized problems: at most
-  // half a wave of tiles) every tile's K loop split over several pairs.  The busiest pair's cost decides.
-  const int max_wide = ceil_div(d_out, kMaxTileW);
+  // ---- column tiling.  Candidates: every projection in tiles of 512 (last one ragged), or with `drop` fewer
+  // wide tiles each and the remaining columns in tiles of w1; or (decode-sized problems: at most half a wave of
+  // tiles, one width) every tile's K loop split over several pairs.  The busiest pair's cost decides.
   long long best = -1;
   const int narrow_widths[3] = {256, 384, 128};
-  for (int n_wide_c = max_wide; n_wide_c >= 0; --n_wide_c) {
-    const int rest = d_out - n_wide_c * kMaxTileW;
+  for (int drop = -1; drop <= max_floor; ++drop) {
     for (int wi = 0; wi < 3; ++wi) {
-      int n_wide = n_wide_c, w0 = kMaxTileW, w1 = narrow_widths[wi];
-      int n_narrow = rest > 0 ? ceil_div(rest, w1) : 0;
-      if (n_wide == 0) { w0 = w1; n_wide = n_narrow; n_narrow = 0; }   // one width only: call it the wide one
-      if (n_wide == 0) continue;
-      if (w0 > d_out) w0 = d_out;                                       // d_out is a multiple of 16
+      int w0 = kMaxTileW, w1 = narrow_widths[wi];
+      int pw[CWL_MAX_GROUP], pn[CWL_MAX_GROUP], n_wide = 0, n_narrow = 0;
+      for (int j = 0; j < n_proj; ++j) {
+        if (drop < 0) { pw[j] = ceil_div(d_out[j], kMaxTileW); pn[j] = 0; }
+        else {
+          pw[j] = d_out[j] / kMaxTileW - drop;
+          if (pw[j] < 0) pw[j] = 0;
+          pn[j] = ceil_div(d_out[j] - pw[j] * kMaxTileW, w1);
+        }
+        n_wide += pw[j]; n_narrow += pn[j];
+      }
+      if (n_wide == 0) {                                                // one width only: call it the wide one
+        w0 = w1; n_wide = n_narrow; n_narrow = 0;
+        for (int j = 0; j < n_proj; ++j) { pw[j] = pn[j]; pn[j] = 0; }
+      }
+      if (w0 > max_dout) w0 = max_dout;                                 // then every projection is a single tile
       const int NW = pl.n_m_pairs * n_wide, NN = pl.n_m_pairs * n_narrow;
       const int used = NW + NN < pairs ? NW + NN : pairs;
       long long worst = 0;
@@ -835,9 +879,10 @@ Plan make_plan(int T, int d_in, int d_out, int R, int pairs, bool allow_split_k,
       if (best < 0 || worst < best) {
         best = worst;
         pl.w0 = w0; pl.n_wide = n_wide; pl.w1 = w1; pl.n_narrow = n_narrow;
+        for (int j = 0; j < n_proj; ++j) { pl.pw[j] = pw[j]; pl.pn[j] = pn[j]; }
         pl.split_k = split_k; pl.kb_per_ksplit = kb_per_ksplit;
       }
-      if (rest <= 0) break;                       // no narrow tiles: their width is irrelevant
+      if (drop < 0) break;                        // no narrow tiles: their width is irrelevant
     }
   }
   const int n_tiles = pl.n_m_pairs * (pl.n_wide + pl.n_narrow);
@@ -851,7 +896,7 @@ Plan make_plan(int T, int d_in, int d_out, int R, int pairs, bool allow_split_k,
 
   pl.boxes = tile_boxes(pl.w0);
   if (pl.n_narrow > 0 && tile_boxes(pl.w1) > pl.boxes) pl.boxes = tile_boxes(pl.w1);
-  if (R > 0 && boxes_for(R / 2) > pl.boxes) pl.boxes = boxes_for(R / 2);
+  if (R > 0 && n_proj * boxes_for(R / 2) > pl.boxes) pl.boxes = n_proj * boxes_for(R / 2);
   pl.stages = kRingBytes / (kABytes + pl.boxes * kBoxBytes);
   if (pl.stages > kMaxStages) pl.stages = kMaxStages;
 
@@ -870,9 +915,10 @@ Plan make_plan(int T, int d_in, int d_out, int R, int pairs, bool allow_split_k,
     for (int want = 1; want <= kMaxSplits; want *= 2) {
       if (want > pl.nkb0) break;
       const int per = ceil_div(pl.nkb0, want), splits = ceil_div(pl.nkb0, per);
-      const size_t scratch = (size_t)T * R * 2 + (size_t)splits * pl.n_m_pairs * 2 * BM * R * 4 + 4096 + 16 * (size_t)pl.n_m_pairs;
+      const size_t RT = (size_t)n_proj * R;
+      const size_t scratch = (size_t)T * RT * 2 + (size_t)splits * pl.n_m_pairs * 2 * BM * RT * 4 + 4096 + 16 * (size_t)pl.n_m_pairs;
       if (scratch_limit > 0 && splits > 1 && scratch > scratch_limit) continue;
-      const long long cs = (long long)per * (16 + 8 * boxes_for(R / 2)) + 176;
+      const long long cs = (long long)per * (16 + 8 * n_proj * boxes_for(R / 2)) + 176;
       const int n_shrink = pl.n_m_pairs * splits;
       uint16_t count[kPairsPlanned];
       long long shrink_time[kPairsPlanned];
@@ -997,11 +1043,12 @@ struct ApplyWorkspace { __nv_bfloat16* Hg; float* partial; float* sk_partial; in
 // Carves the workspace for a plan.
 size_t carve_apply(ApplyWorkspace& w, char* base, const Plan& pl, int T, int R) {
   auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  const size_t RT = (size_t)pl.n_proj * R;
   size_t off = 0;
   w.Hg = reinterpret_cast<__nv_bfloat16*>(base ? base + off : nullptr);
-  if (R > 0) off = up(off + (size_t)T * R * sizeof(__nv_bfloat16));
+  if (R > 0) off = up(off + (size_t)T * RT * sizeof(__nv_bfloat16));
   w.partial = reinterpret_cast<float*>(base ? base + off : nullptr);
-  if (R > 0 && pl.shrink_splits > 1) off = up(off + (size_t)pl.shrink_splits * pl.n_m_pairs * 2 * BM * R * sizeof(float));
+  if (R > 0 && pl.shrink_splits > 1) off = up(off + (size_t)pl.shrink_splits * pl.n_m_pairs * 2 * BM * RT * sizeof(float));
   w.sk_partial = reinterpret_cast<float*>(base ? base + off : nullptr);
   const bool split = pl.split_k > 1;
   const size_t n_tiles = (size_t)pl.n_m_pairs * pl.n_wide;              // split plans have one tile width
@@ -1013,55 +1060,80 @@ size_t carve_apply(ApplyWorkspace& w, char* base, const Plan& pl, int T, int R) 
   return off < 256 ? 256 : off;
 }
 
-cwl_status apply_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, const void* A, int64_t lda,
-                      const void* B, int64_t ldb, int32_t T, int32_t d_in, int32_t d_out, int32_t R,
-                      cwl_chunk_table table, int32_t window, void* Y, int64_t ldy, void* workspace,
-                      size_t workspace_bytes, int32_t* status_word, void* stream_, bool allow_split_k,
-                      size_t scratch_limit = 0) {
-  if (T < 0 || d_in < 1 || d_out < 1 || R < 0 || window < 0) return CWL_ERR_INVALID_ARG;
-  if (T > 0 && (X == nullptr || Y == nullptr)) return CWL_ERR_INVALID_ARG;
-  if (W == nullptr) return CWL_ERR_INVALID_ARG;
-  const bool adapter = (A != nullptr && B != nullptr && R > 0);
-  if (d_in % 16 != 0 || d_out % 16 != 0) return CWL_ERR_UNSUPPORTED;
-  if (adapter && (R % 16 != 0 || R > CWL_MAX_RANK)) return CWL_ERR_UNSUPPORTED;
-  if (ldx < d_in || ldw < d_out || ldy < d_out || (adapter && (lda < R || ldb < d_out))) return CWL_ERR_SHAPE;
-  if (ldx % 8 != 0 || ldw % 8 != 0 || ldy % 8 != 0 || (adapter && (lda % 8 != 0 || ldb % 8 != 0))) return CWL_ERR_SHAPE;
-  if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || (adapter && (!aligned16(A) || !aligned16(B))))
-    return CWL_ERR_SHAPE;
+// Argument checks shared by every entry point.  `adapter` comes back true when every projection has both factors.
+cwl_status check_group(const void* X, int64_t ldx, const cwl_projection* proj, int n_proj, int T, int d_in, int R,
+                       const cwl_chunk_table& table, int window, bool& adapter) {
+  if (proj == nullptr || n_proj < 1 || n_proj > CWL_MAX_GROUP) return CWL_ERR_INVALID_ARG;
+  if (T < 0 || d_in < 1 || R < 0 || window < 0) return CWL_ERR_INVALID_ARG;
+  if (T > 0 && X == nullptr) return CWL_ERR_INVALID_ARG;
+  int with = 0;
+  for (int j = 0; j < n_proj; ++j) {
+    if (proj[j].d_out < 1 || proj[j].W == nullptr || (T > 0 && proj[j].Y == nullptr)) return CWL_ERR_INVALID_ARG;
+    if (proj[j].A != nullptr && proj[j].B != nullptr && R > 0) ++with;
+  }
+  if (with != 0 && with != n_proj) return CWL_ERR_INVALID_ARG;   // adapters on all projections of a group or on none
+  adapter = with == n_proj;
+  if (d_in % 16 != 0) return CWL_ERR_UNSUPPORTED;
+  if (adapter && (R % 16 != 0 || R > CWL_MAX_RANK || n_proj * R > kMaxTileW)) return CWL_ERR_UNSUPPORTED;
+  if (ldx < d_in || ldx % 8 != 0 || !aligned16(X)) return CWL_ERR_SHAPE;
+  for (int j = 0; j < n_proj; ++j) {
+    const cwl_projection& q = proj[j];
+    if (q.d_out % 16 != 0) return CWL_ERR_UNSUPPORTED;
+    if (q.ldw < q.d_out || q.ldy < q.d_out || (adapter && (q.lda < R || q.ldb < q.d_out))) return CWL_ERR_SHAPE;
+    if (q.ldw % 8 != 0 || q.ldy % 8 != 0 || (adapter && (q.lda % 8 != 0 || q.ldb % 8 != 0))) return CWL_ERR_SHAPE;
+    if (!aligned16(q.W) || !aligned16(q.Y) || (adapter && (!aligned16(q.A) || !aligned16(q.B)))) return CWL_ERR_SHAPE;
+  }
   if (adapter && (table.offsets == nullptr || table.rank == nullptr || table.scale == nullptr ||
                   table.flags == nullptr || table.n_chunks == nullptr || table.capacity < 0))
     return CWL_ERR_INVALID_ARG;
+  return CWL_OK;
+}
+
+// Plans, carves the workspace, builds the tensor maps and launches one fused kernel for a group of projections.
+cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* proj, int n_proj, int32_t T,
+                            int32_t d_in, int32_t R, cwl_chunk_table table, int32_t window, void* workspace,
+                            size_t workspace_bytes, int32_t* status_word, void* stream_, bool allow_split_k,
+                            size_t scratch_limit) {
+  bool adapter = false;
+  const cwl_status chk = check_group(X, ldx, proj, n_proj, T, d_in, R, table, window, adapter);
+  if (chk != CWL_OK) return chk;
   if (T == 0) return CWL_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   const int Reff = adapter ? R : 0;
+  int d_out[CWL_MAX_GROUP];
+  for (int j = 0; j < n_proj; ++j) d_out[j] = proj[j].d_out;
 
   ApplyWorkspace ws{nullptr, nullptr, nullptr, nullptr, 0};
-  Plan pl = make_plan(T, d_in, d_out, Reff, max_pairs(), allow_split_k, scratch_limit);
+  Plan pl = make_plan(T, d_in, n_proj, d_out, Reff, max_pairs(), allow_split_k, scratch_limit);
   const size_t need = carve_apply(ws, static_cast<char*>(workspace), pl, T, Reff);
   const bool have_ws = workspace != nullptr && workspace_bytes >= need && (reinterpret_cast<uintptr_t>(workspace) & 255u) == 0;
   if (!have_ws && !adapter && pl.split_k > 1) {
     // the plain projection needs scratch only when its K loop is split; without a workspace it runs unsplit
-    pl = make_plan(T, d_in, d_out, Reff, max_pairs(), false, scratch_limit);
+    pl = make_plan(T, d_in, n_proj, d_out, Reff, max_pairs(), false, scratch_limit);
   } else if (!have_ws && (adapter || pl.split_k > 1)) {
     return CWL_ERR_WORKSPACE;
   }
 
-  CUtensorMap mX, mW, mA, mH, mB, mY;
-  if (!make_map(&mY, Y, (uint64_t)d_out, (uint64_t)T, (uint64_t)ldy, 64, 32)) return CWL_ERR_CUDA;
-  if (!make_map(&mX, X, (uint64_t)d_in, (uint64_t)T, (uint64_t)ldx, BK, BM)) return CWL_ERR_CUDA;
-  if (!make_map(&mW, W, (uint64_t)d_out, (uint64_t)d_in, (uint64_t)ldw, kBoxCols, BK)) return CWL_ERR_CUDA;
-  if (adapter) {
-    if (!make_map(&mA, A, (uint64_t)R, (uint64_t)d_in, (uint64_t)lda, kBoxCols, BK)) return CWL_ERR_CUDA;
-    if (!make_map(&mH, ws.Hg, (uint64_t)R, (uint64_t)T, (uint64_t)R, BK, BM)) return CWL_ERR_CUDA;
-    if (!make_map(&mB, B, (uint64_t)d_out, (uint64_t)R, (uint64_t)ldb, kBoxCols, BK)) return CWL_ERR_CUDA;
-  } else {
-    mA = mW; mH = mX; mB = mW;   // never dereferenced when R == 0
+  GroupMaps maps;
+  memset(&maps, 0, sizeof(maps));
+  if (!make_map(&maps.x, X, (uint64_t)d_in, (uint64_t)T, (uint64_t)ldx, BK, BM)) return CWL_ERR_CUDA;
+  maps.h = maps.x;                                  // never dereferenced when R == 0
+  if (adapter && !make_map(&maps.h, ws.Hg, (uint64_t)n_proj * R, (uint64_t)T, (uint64_t)n_proj * R, BK, BM)) return CWL_ERR_CUDA;
+  for (int j = 0; j < n_proj; ++j) {
+    const cwl_projection& q = proj[j];
+    if (!make_map(&maps.y[j], q.Y, (uint64_t)q.d_out, (uint64_t)T, (uint64_t)q.ldy, 64, 32)) return CWL_ERR_CUDA;
+    if (!make_map(&maps.w[j], q.W, (uint64_t)q.d_out, (uint64_t)d_in, (uint64_t)q.ldw, kBoxCols, BK)) return CWL_ERR_CUDA;
+    maps.a[j] = maps.w[j]; maps.b[j] = maps.w[j];   // never dereferenced when R == 0
+    if (adapter) {
+      if (!make_map(&maps.a[j], q.A, (uint64_t)R, (uint64_t)d_in, (uint64_t)q.lda, kBoxCols, BK)) return CWL_ERR_CUDA;
+      if (!make_map(&maps.b[j], q.B, (uint64_t)q.d_out, (uint64_t)R, (uint64_t)q.ldb, kBoxCols, BK)) return CWL_ERR_CUDA;
+    }
   }
 
   ApplyParams p{};
-  p.T = T; p.d_in = d_in; p.d_out = d_out; p.R = Reff;
+  p.T = T; p.d_in = d_in; p.R = Reff; p.RT = n_proj * Reff;
   p.window = window;
-  p.Y = static_cast<__nv_bfloat16*>(Y); p.ldy = ldy;
+  for (int j = 0; j < n_proj; ++j) { p.Y[j] = static_cast<__nv_bfloat16*>(proj[j].Y); p.ldy[j] = proj[j].ldy; }
   p.Hg = ws.Hg; p.partial = ws.partial; p.sk_partial = ws.sk_partial;
   p.counters = ws.sync; p.flags = ws.sync + 2 * pl.n_m_pairs; p.sk_counters = ws.sync + 4 * pl.n_m_pairs;
   p.table = table; p.status_word = status_word;
@@ -1077,9 +1149,22 @@ cwl_status apply_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, co
     CWL_CUDA_TRY(cudaFuncSetAttribute(apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout::kTotal));
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
-  apply_kernel<<<2 * pl.pairs, kThreads, SmemLayout::kTotal, stream>>>(mX, mW, mA, mH, mB, mY, p);
+  apply_kernel<<<2 * pl.pairs, kThreads, SmemLayout::kTotal, stream>>>(maps, p);
   CWL_CUDA_TRY(cudaGetLastError());
   return CWL_OK;
+}
+
+cwl_status apply_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, const void* A, int64_t lda,
+                      const void* B, int64_t ldb, int32_t T, int32_t d_in, int32_t d_out, int32_t R,
+                      cwl_chunk_table table, int32_t window, void* Y, int64_t ldy, void* workspace,
+                      size_t workspace_bytes, int32_t* status_word, void* stream, bool allow_split_k,
+                      size_t scratch_limit = 0) {
+  const bool adapter = (A != nullptr && B != nullptr && R > 0);
+  cwl_projection q;
+  q.W = W; q.ldw = ldw; q.A = adapter ? A : nullptr; q.lda = lda; q.B = adapter ? B : nullptr; q.ldb = ldb;
+  q.Y = Y; q.ldy = ldy; q.d_out = d_out;
+  return apply_group_impl(X, ldx, &q, 1, T, d_in, R, table, window, workspace, workspace_bytes, status_word, stream,
+                          allow_split_k, scratch_limit);
 }
 
 }  // namespace
@@ -1088,7 +1173,7 @@ cwl_status apply_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, co
 extern "C" size_t cwl_apply_workspace_bytes(int32_t T, int32_t d_in, int32_t d_out, int32_t R) {
   if (T <= 0 || d_in <= 0 || d_out <= 0 || R < 0) return 256;
   cwl::ApplyWorkspace w;
-  const cwl::Plan pl = cwl::make_plan(T, d_in, d_out, R, cwl::max_pairs(), true);
+  const cwl::Plan pl = cwl::make_plan(T, d_in, 1, &d_out, R, cwl::max_pairs(), true);
   return cwl::carve_apply(w, nullptr, pl, T, R);
 }
 
@@ -1096,7 +1181,7 @@ extern "C" cwl_status cwl_apply_plan(int32_t T, int32_t d_in, int32_t d_out, int
                                      cwl_apply_plan_info* out) {
   if (out == nullptr || T < 1 || d_in < 16 || d_out < 16 || R < 0 || pairs < 1) return CWL_ERR_INVALID_ARG;
   if (d_in % 16 != 0 || d_out % 16 != 0 || R % 16 != 0 || R > CWL_MAX_RANK) return CWL_ERR_UNSUPPORTED;
-  const cwl::Plan pl = cwl::make_plan(T, d_in, d_out, R, pairs, true);
+  const cwl::Plan pl = cwl::make_plan(T, d_in, 1, &d_out, R, pairs, true);
   out->pairs = pl.pairs; out->row_tiles = pl.n_m_pairs;
   out->wide_width = pl.w0; out->wide_tiles_per_row = pl.n_wide;
   out->narrow_width = pl.n_narrow > 0 ? pl.w1 : 0; out->narrow_tiles_per_row = pl.n_narrow;
@@ -1118,6 +1203,23 @@ extern "C" cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64
                                 int32_t* status_word, void* stream) {
   return cwl::apply_impl(X, ldx, W, ldw, A, lda, B, ldb, T, d_in, d_out, R, table, window, Y, ldy, workspace,
                          workspace_bytes, status_word, stream, true);
+}
+
+extern "C" size_t cwl_apply_grouped_workspace_bytes(int32_t T, int32_t d_in, int32_t n_proj, const int32_t* d_out,
+                                                    int32_t R) {
+  if (T <= 0 || d_in <= 0 || R < 0 || d_out == nullptr || n_proj < 1 || n_proj > CWL_MAX_GROUP) return 256;
+  int widths[CWL_MAX_GROUP];
+  for (int j = 0; j < n_proj; ++j) { if (d_out[j] < 1) return 256; widths[j] = d_out[j]; }
+  cwl::ApplyWorkspace w;
+  const cwl::Plan pl = cwl::make_plan(T, d_in, n_proj, widths, R, cwl::max_pairs(), true);
+  return cwl::carve_apply(w, nullptr, pl, T, R);
+}
+
+extern "C" cwl_status cwl_apply_grouped(const void* X, int64_t ldx, const cwl_projection* proj, int32_t n_proj,
+                                        int32_t T, int32_t d_in, int32_t R, cwl_chunk_table table, int32_t window,
+                                        void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream) {
+  return cwl::apply_group_impl(X, ldx, proj, n_proj, T, d_in, R, table, window, workspace, workspace_bytes,
+                               status_word, stream, true, 0);
 }
 
 // ------------------------------------------------------------------------------ no-allocation variant
@@ -1154,7 +1256,7 @@ cwl_status noalloc_scratch(void** out) {
 extern "C" size_t cwl_apply_noalloc_scratch_need(int32_t T, int32_t d_in, int32_t d_out, int32_t R) {
   if (T <= 0 || d_in <= 0 || d_out <= 0 || R < 0) return 256;
   cwl::ApplyWorkspace w;
-  const cwl::Plan pl = cwl::make_plan(T, d_in, d_out, R, cwl::max_pairs(), false, CWL_NOALLOC_SCRATCH_BYTES);
+  const cwl::Plan pl = cwl::make_plan(T, d_in, 1, &d_out, R, cwl::max_pairs(), false, CWL_NOALLOC_SCRATCH_BYTES);
   return cwl::carve_apply(w, nullptr, pl, T, R);
 }
 
