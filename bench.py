@@ -45,7 +45,7 @@ def load_peaks():
 
 # Revision tag of the dominant kernel the ncu counters under profiles/ were taken on.  Bump it whenever
 # cwl_apply's kernel changes: a traffic figure taken on another revision is reported as null.
-APPLY_KERNEL_REVISION = "pairs-256x512-planned-tma-store"
+APPLY_KERNEL_REVISION = "pairs-256x512-grouped"
 
 
 def load_traffic(key: str):
@@ -237,7 +237,7 @@ def run_ours(args):
 
     w = make_workload(args.workload)
     n_layers = args.layers if args.workload == "cfg5" else 1
-    hp = HotPath(w, n_layers=n_layers)
+    hp = HotPath(w, n_layers=n_layers, grouped=not args.no_group)
     stream = torch.cuda.current_stream()
 
     # thresholds of the rule-based percentile mapping (Sec. IV-C): quartiles of this batch's scores
@@ -385,7 +385,7 @@ def run_ours(args):
     roof["frac_of_nominal_2250"] = (f_alg / (apply_avg_ms * 1e-3) / 1e12) / 2250.0
 
     parts = (["score"] if hp.logits is not None else []) + ([] if hp.fixed_table else ["partition"]) + \
-        [f"{len(hp.projs)} x apply"]
+        [f"{len(hp.projs)} projections in {len(hp.launch_groups())} apply launches"]
     steps_include = (f"{n_layers} layers x (" if n_layers > 1 else "(") + " + ".join(parts) + ")"
     step_bytes = n_layers * (sum(2 * p.d_in * p.d_out for p in hp.projs) +
                              (hp.logits.numel() * 4 if hp.logits is not None else 0))
@@ -431,6 +431,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--layers", type=int, default=32, help="layers of the cfg5 projection stack (a step runs all of them)")
+    ap.add_argument("--no-group", action="store_true",
+                    help="one cwl_apply launch per projection instead of grouped launches for q,k,v and gate,up")
     ap.add_argument("--lean", action="store_true",
                     help="timed region only (no comparison runs, end-to-end leg or CPU baseline): for profiler runs")
     args = ap.parse_args()

@@ -443,8 +443,12 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
-    if (lane == 0) {
+    // The whole warp walks the ring; per K block lane 0 arms the barrier and loads the left operand, lanes 1..n
+    // load one right-operand box each, so the copies of a step go out with one instruction instead of a chain.
+    {
       uint32_t it_cnt = 0;      // running stage counter across items
+      uint32_t s = 0, ph = 0;   // ring slot and phase parity of it_cnt, kept incrementally (no division per step)
+      const uint32_t leader_full0 = mapa_shared(full_bar(0), 0);   // full_bar(0) in the leader's shared memory
       bool ok = true;
       Item item;
       for (int i = 0; ok && get_item(i, pair, sh_begin, p, item); ++i) {
@@ -456,36 +460,42 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
         const int boxes_a = boxes_for(ca), boxes_b = boxes_for(cb);
         const int col_a = shrink ? (int)rank * ca : item.n0 + (int)rank * ca;
         const int col_b = item.n0 + item.wa + (int)rank * cb;
-        const int n_right = shrink ? pl.n_proj : 1;           // matrices the first group of boxes comes from
-        const uint32_t tx_pair = 2u * (kABytes + (n_right * boxes_a + boxes_b) * kBoxBytes);
+        const int n_boxes = shrink ? pl.n_proj * boxes_a : boxes_a + boxes_b;
+        const uint32_t tx_pair = 2u * (kABytes + n_boxes * kBoxBytes);
+        // this lane's box (lanes 1..n_boxes): source matrix in the d_in blocks and in the R blocks, column, slot
+        const int bi = lane - 1;
+        const bool has_box = bi >= 0 && bi < n_boxes;
+        const CUtensorMap* map0 = &tm.w[item.proj];
+        const CUtensorMap* map1 = &tm.b[item.proj];
+        int box_x = 0;
+        if (has_box) {
+          if (shrink) { map0 = &tm.a[bi / boxes_a]; box_x = col_a + (bi % boxes_a) * kBoxCols; }
+          else box_x = bi < boxes_a ? col_a + bi * kBoxCols : col_b + (bi - boxes_a) * kBoxCols;
+        }
         const int n_blk = item.n_blk0 + item.n_blk1;
         for (int b = 0; b < n_blk; ++b, ++it_cnt) {
-          const int s = it_cnt % n_stages;
-          const uint32_t ph = (it_cnt / n_stages) & 1u;
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+          bool step_ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag);
           const bool phase1 = b >= item.n_blk0;
           if (phase1 && b == item.n_blk0) {
             // H' of this CTA's row tile must have been published by whoever finished its shrink
-            if (!wait_word(p.flags + m_tile, 1, abort_flag)) { ok = false; break; }
+            if (lane == 0 && step_ok) step_ok = wait_word(p.flags + m_tile, 1, abort_flag);
             fence_proxy_async();
           }
+          if (!__all_sync(0xffffffffu, step_ok)) { ok = false; break; }
           const int k = phase1 ? (b - item.n_blk0) * BK : (item.kb0 + b) * BK;
           const uint32_t sa = base + s * stage_bytes, sb = sa + kABytes;
-          const uint32_t leader_full = mapa_shared(full_bar(s), 0); // the same barrier in the leader's shared memory
-          if (rank == 0) mbar_expect_tx(full_bar(s), tx_pair);
-          if (phase1) tma_load_2d_pair(sa, &tm.h, leader_full, item.proj * p.R + k, m_tile * BM);
-          else tma_load_2d_pair(sa, &tm.x, leader_full, k, m_tile * BM);
-          for (int q = 0; q < n_right; ++q) {
-            const CUtensorMap* right = shrink ? &tm.a[q] : (phase1 ? &tm.b[item.proj] : &tm.w[item.proj]);
-            for (int j = 0; j < boxes_a; ++j)
-              tma_load_2d_pair(sb + (q * boxes_a + j) * kBoxBytes, right, leader_full, col_a + j * kBoxCols, k);
+          const uint32_t leader_full = leader_full0 + 8u * s;      // this stage's barrier in the leader's shared memory
+          if (lane == 0) {
+            if (rank == 0) mbar_expect_tx(full_bar(s), tx_pair);
+            if (phase1) tma_load_2d_pair(sa, &tm.h, leader_full, item.proj * p.R + k, m_tile * BM);
+            else tma_load_2d_pair(sa, &tm.x, leader_full, k, m_tile * BM);
+          } else if (has_box) {
+            tma_load_2d_pair(sb + bi * kBoxBytes, phase1 ? map1 : map0, leader_full, box_x, k);
           }
-          const CUtensorMap* right = phase1 ? &tm.b[item.proj] : &tm.w[item.proj];
-          for (int j = 0; j < boxes_b; ++j)
-            tma_load_2d_pair(sb + (boxes_a + j) * kBoxBytes, right, leader_full, col_b + j * kBoxCols, k);
+          if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
         }
       }
-      if (!ok && rank == 0) {
+      if (!ok && rank == 0 && lane == 0) {
         // drain: give the copies already issued a bounded chance to land before the CTA leaves
         for (uint32_t back = 1; back <= (uint32_t)n_stages && back <= it_cnt; ++back) {
           const uint32_t j = it_cnt - back;
@@ -497,7 +507,8 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
     if (lane == 0 && rank == 0) {
-      uint32_t it_cnt = 0, local = 0;
+      uint32_t local = 0;
+      uint32_t s = 0, ph = 0;   // ring slot and phase parity, kept incrementally
       bool ok = true;
       Item item;
       for (int i = 0; ok && get_item(i, pair, sh_begin, p, item); ++i, ++local) {
@@ -509,9 +520,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
         if (!mbar_wait(acc_empty_bar, (local & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const int n_blk = item.n_blk0 + item.n_blk1;
-        for (int b = 0; b < n_blk; ++b, ++it_cnt) {
-          const int s = it_cnt % n_stages;
-          const uint32_t ph = (it_cnt / n_stages) & 1u;
+        for (int b = 0; b < n_blk; ++b) {
           if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const bool phase1 = b >= item.n_blk0;
@@ -535,6 +544,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
             }
           }
           umma_commit_pair(empty_bar(s));            // frees the stage in both CTAs once these MMAs have read it
+          if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
         }
         if (ok) umma_commit_pair(acc_full_bar);      // accumulator complete, both CTAs
       }
@@ -809,8 +819,8 @@ int shrink_splits_for(int T, int d_in) {
 // Chooses tile widths, the K split and who does the shrink work for `pairs` resident CTA pairs.
 // Depends on the shape and on `pairs` only.  allow_split_k = false keeps every tile whole; scratch_limit > 0
 // keeps the shrink's split small enough for H' and the partial sums to fit that many bytes (one split always may).
-Plan make_plan(int T, int d_in, int n_proj, const int* d_out, int R, int pairs, bool allow_split_k,
-               size_t scratch_limit = 0) {
+Plan search_plan(int T, int d_in, int n_proj, const int* d_out, int R, int pairs, bool allow_split_k,
+                 size_t scratch_limit) {
   Plan pl;
   memset(&pl, 0, sizeof(pl));
   if (pairs > kPairsPlanned) pairs = kPairsPlanned;
@@ -918,15 +928,23 @@ Plan make_plan(int T, int d_in, int n_proj, const int* d_out, int R, int pairs, 
       const size_t RT = (size_t)n_proj * R;
       const size_t scratch = (size_t)T * RT * 2 + (size_t)splits * pl.n_m_pairs * 2 * BM * RT * 4 + 4096 + 16 * (size_t)pl.n_m_pairs;
       if (scratch_limit > 0 && splits > 1 && scratch > scratch_limit) continue;
-      const long long cs = (long long)per * (16 + 8 * n_proj * boxes_for(R / 2)) + 176;
+      // measured: a shrink K block costs about 1.3x its staged bytes (narrow MMAs), an item ~4 us of fixed cost
+      const long long cs = (long long)per * (16 + 8 * n_proj * boxes_for(R / 2)) * 13 / 10 + 250;
+      const long long due = first_tile * 4 / 5;
       const int n_shrink = pl.n_m_pairs * splits;
       uint16_t count[kPairsPlanned];
       long long shrink_time[kPairsPlanned];
       for (int g = 0; g < pl.pairs; ++g) { load[g] = base_load[g]; count[g] = 0; shrink_time[g] = 0; }
       for (int i = 0; i < n_shrink; ++i) {
-        int at = pl.pairs - 1;
+        // the lightest pair whose shrink work still ends before H' is due; failing that, the one that ends first
+        int at = -1;
         for (int g = pl.pairs - 1; g >= 0; --g)
-          if (load[g] < load[at]) at = g;
+          if (shrink_time[g] + cs <= due && (at < 0 || load[g] < load[at])) at = g;
+        if (at < 0) {
+          at = pl.pairs - 1;
+          for (int g = pl.pairs - 1; g >= 0; --g)
+            if (shrink_time[g] < shrink_time[at] || (shrink_time[g] == shrink_time[at] && load[g] < load[at])) at = g;
+        }
         load[at] += cs; shrink_time[at] += cs; count[at]++;
       }
       long long worst = 0, latest = 0;
@@ -934,8 +952,7 @@ Plan make_plan(int T, int d_in, int n_proj, const int* d_out, int R, int pairs, 
         if (load[g] > worst) worst = load[g];
         if (shrink_time[g] > latest) latest = shrink_time[g];
       }
-      const long long due = first_tile * 4 / 5;
-      const long long total = worst + (latest > due ? latest - due : 0);
+      const long long total = worst + (latest > due ? 2 * (latest - due) : 0);
       if (best_total < 0 || total < best_total) {
         best_total = total;
         pl.shrink_splits = splits; pl.kb_per_split = per;
@@ -949,6 +966,32 @@ Plan make_plan(int T, int d_in, int n_proj, const int* d_out, int R, int pairs, 
   pl.makespan = 0;
   for (int g = 0; g < pl.pairs; ++g)
     if (load[g] > pl.makespan) pl.makespan = load[g];
+  return pl;
+}
+
+// The search costs tens of microseconds of host time, as much as a small launch: plans are remembered per shape.
+Plan make_plan(int T, int d_in, int n_proj, const int* d_out, int R, int pairs, bool allow_split_k,
+               size_t scratch_limit = 0) {
+  struct Key { int v[6 + CWL_MAX_GROUP]; unsigned long long limit; };
+  struct Entry { Key key; Plan plan; };
+  static std::mutex mu;
+  static Entry entries[64];
+  static int n_entries = 0, next_slot = 0;
+  Key key;
+  memset(&key, 0, sizeof(key));
+  key.v[0] = T; key.v[1] = d_in; key.v[2] = n_proj; key.v[3] = R; key.v[4] = pairs; key.v[5] = allow_split_k ? 1 : 0;
+  for (int j = 0; j < n_proj && j < CWL_MAX_GROUP; ++j) key.v[6 + j] = d_out[j];
+  key.limit = scratch_limit;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < n_entries; ++i)
+      if (memcmp(&entries[i].key, &key, sizeof(Key)) == 0) return entries[i].plan;
+  }
+  const Plan pl = search_plan(T, d_in, n_proj, d_out, R, pairs, allow_split_k, scratch_limit);
+  std::lock_guard<std::mutex> lock(mu);
+  entries[next_slot].key = key; entries[next_slot].plan = pl;
+  next_slot = (next_slot + 1) % 64;
+  if (n_entries < 64) ++n_entries;
   return pl;
 }
 

@@ -35,7 +35,9 @@ def policy_struct(p: Policy) -> cwl.CPolicy:
 class HotPath:
     """Device-resident state of one layer's adapted projections plus the scheduler in front."""
 
-    def __init__(self, w: Workload, device: str = "cuda", keep_host: bool = False, n_layers: int = 1):
+    def __init__(self, w: Workload, device: str = "cuda", keep_host: bool = False, n_layers: int = 1,
+                 grouped: bool = True):
+        self.grouped = grouped
         self.T, self.R, self.policy = w.T, w.R, w.policy
         self.device = device
         self.cu_seqlens = torch.from_numpy(w.cu_seqlens).to(device)
@@ -64,6 +66,10 @@ class HotPath:
         self.fixed_table = w.table is not None
         self.part_ws = torch.empty(cwl.cwl_partition_workspace_bytes(w.T, self.n_seq), dtype=torch.uint8, device=device)
         ws_bytes = max(cwl.cwl_apply_workspace_bytes(w.T, p.d_in, p.d_out, w.R) for p in w.projections)
+        for group in self.launch_groups():
+            if len(group) > 1:
+                ws_bytes = max(ws_bytes, cwl.cwl_apply_grouped_workspace_bytes(
+                    w.T, group[0].d_in, [q.d_out for q in group], w.R))
         self.apply_ws = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
         self.cpolicy = policy_struct(w.policy)
@@ -85,11 +91,37 @@ class HotPath:
         cwl.cwl_partition(self.score, self.cu_seqlens, self.cpolicy, table=self.table, workspace=self.part_ws,
                           status_word=self.status)
 
+    # projections that read the same activation go out as one grouped launch where that is measured to pay:
+    # gate + up (2 x 11008 columns fill the tile waves better together).  q, k, v grouped run faster without an
+    # adapter but slower with one (their joint shrink delays the first wave of tiles), so they stay separate.
+    GROUPS = (("gate", "up"),)
+    GROUP_MIN_T = 512           # below this a call is decode-sized: separate calls, whose K loop is split
+
+    def launch_groups(self, layer: int = 0) -> List[List[DeviceProjection]]:
+        projs = self.layers[layer]
+        if not self.grouped or self.T < self.GROUP_MIN_T:
+            return [[p] for p in projs]
+        by_name = {p.name: p for p in projs}
+        out, used = [], set()
+        for p in projs:
+            if p.name in used:
+                continue
+            members = next((g for g in self.GROUPS if p.name in g and all(n in by_name for n in g)), (p.name,))
+            out.append([by_name[n] for n in members])
+            used.update(members)
+        return out
+
     def apply_step(self, table: Optional[cwl.DeviceChunkTable] = None, dense: bool = False, layer: int = 0) -> None:
         tab = table if table is not None else self.table
-        for p in self.layers[layer]:
-            cwl.cwl_apply(self.X[p.d_in], p.W, None if dense else p.A, None if dense else p.B, tab,
-                          self.policy.window, Y=p.Y, workspace=self.apply_ws, status_word=self.status)
+        for group in self.launch_groups(layer):
+            p = group[0]
+            if len(group) == 1:
+                cwl.cwl_apply(self.X[p.d_in], p.W, None if dense else p.A, None if dense else p.B, tab,
+                              self.policy.window, Y=p.Y, workspace=self.apply_ws, status_word=self.status)
+            else:
+                cwl.cwl_apply_grouped(self.X[p.d_in], [q.W for q in group], None if dense else [q.A for q in group],
+                                      None if dense else [q.B for q in group], tab, self.policy.window,
+                                      Ys=[q.Y for q in group], workspace=self.apply_ws, status_word=self.status)
 
     def step(self) -> None:
         """One pass of the whole hot path on the current stream (no host synchronisation)."""
@@ -101,7 +133,7 @@ class HotPath:
             self.apply_step(layer=layer)
 
     def launches_per_step(self) -> int:
-        n = self.LAUNCHES_APPLY * len(self.projs)
+        n = self.LAUNCHES_APPLY * len(self.launch_groups())
         if self.logits is not None:
             n += self.LAUNCHES_SCORE
         if not self.fixed_table:
