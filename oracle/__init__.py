@@ -198,3 +198,59 @@ def apply(X: np.ndarray, W: np.ndarray, A: Optional[np.ndarray], B: Optional[np.
     if rc != 0:
         raise ValueError(f"cwlo_apply: status {rc}")
     return Y
+
+
+# ------------------------------------------------------------------ decode-time scheduler (streaming)
+STREAM_MAX_MIN_LEN = 64
+
+
+class _StreamState(C.Structure):
+    _fields_ = [("pos", C.c_int32), ("len", C.c_int32), ("cur_rung", C.c_int32), ("prev_rung", C.c_int32),
+                ("hi_used", C.c_int32), ("first", C.c_int32), ("ring", C.c_int64 * STREAM_MAX_MIN_LEN)]
+
+
+class RowGate(C.Structure):
+    _fields_ = [("rank_in", C.c_int32), ("rank_out", C.c_int32), ("scale_in", C.c_float), ("scale_out", C.c_float),
+                ("lambda_", C.c_float), ("pos_in_chunk", C.c_int32), ("opened", C.c_int32)]
+
+
+ROW_GATE_DTYPE = np.dtype([("rank_in", np.int32), ("rank_out", np.int32), ("scale_in", np.float32),
+                           ("scale_out", np.float32), ("lam", np.float32), ("pos_in_chunk", np.int32),
+                           ("opened", np.int32)])
+
+
+class Stream:
+    """Decode-time scheduler of ONE sequence (Sec. III-B "grouped online", state cached across steps)."""
+
+    def __init__(self, ranks, scales, thresholds, min_len, max_len, window, hi_budget=-1):
+        self.policy = _policy_struct(ranks, scales, thresholds, min_len, max_len, window, hi_budget)
+        self.state = _StreamState()
+        lib().cwlo_stream_reset(C.byref(self.state))
+
+    def step(self, score: float) -> np.void:
+        g = RowGate()
+        rc = lib().cwlo_stream_step(C.byref(self.state), C.c_float(float(score)), C.byref(self.policy), C.byref(g))
+        if rc != 0:
+            raise ValueError(f"cwlo_stream_step: status {rc}")
+        out = np.zeros((), dtype=ROW_GATE_DTYPE)
+        out["rank_in"], out["rank_out"], out["scale_in"], out["scale_out"] = g.rank_in, g.rank_out, g.scale_in, g.scale_out
+        out["lam"], out["pos_in_chunk"], out["opened"] = g.lambda_, g.pos_in_chunk, g.opened
+        return out
+
+
+def apply_rows(X: np.ndarray, W: np.ndarray, A: np.ndarray, B: np.ndarray, gates: np.ndarray) -> np.ndarray:
+    """Adapted projection in fp64 with one (rank_in, scale_in, rank_out, scale_out, lambda) descriptor per row.
+    ``gates`` is a structured array of ROW_GATE_DTYPE."""
+    X = np.ascontiguousarray(X, dtype=np.uint16); W = np.ascontiguousarray(W, dtype=np.uint16)
+    A = np.ascontiguousarray(A, dtype=np.uint16); B = np.ascontiguousarray(B, dtype=np.uint16)
+    gates = np.ascontiguousarray(gates, dtype=ROW_GATE_DTYPE)
+    T, d_in = X.shape
+    d_out, R = W.shape[1], A.shape[1]
+    assert gates.shape == (T,) and ROW_GATE_DTYPE.itemsize == C.sizeof(RowGate)
+    Y = np.empty((T, d_out), dtype=np.float64)
+    rc = lib().cwlo_apply_rows(_ptr(X), C.c_int64(d_in), _ptr(W), C.c_int64(d_out), _ptr(A), C.c_int64(R),
+                               _ptr(B), C.c_int64(d_out), C.c_int32(T), C.c_int32(d_in), C.c_int32(d_out), C.c_int32(R),
+                               gates.ctypes.data_as(C.c_void_p), _ptr(Y), C.c_int64(d_out))
+    if rc != 0:
+        raise ValueError(f"cwlo_apply_rows: status {rc}")
+    return Y

@@ -276,3 +276,100 @@ int cwlo_apply(const uint16_t* X, int64_t ldx, const uint16_t* W, int64_t ldw,
   }
   return bad ? CWLO_ERR_ARG : CWLO_OK;
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * Decode-time scheduler (Sec. III-A "streaming and cached", III-B "grouped online", III-F "the
+ * scheduler's state is cached across steps").  The paper names the constraints only; the rule is
+ * this build's causal reading: a token may open a new chunk only on what has been seen so far.
+ *
+ * Per sequence: the open chunk's length and the rung it was opened on (a chunk's configuration is
+ * fixed while it is open), the previous chunk's rung, and the quantised scores of the last L_min
+ * tokens.  On a new token with quantised score q:
+ *   1. q enters the trailing window (the last min(L_min, tokens seen) scores, the new one included);
+ *   2. the first token of a sequence opens the first chunk on the rung of that window;
+ *   3. otherwise, if the open chunk holds at least L_min tokens and either holds L_max of them or
+ *      the window's rung differs from the open chunk's rung, the token opens a new chunk on the
+ *      window's rung (with a budget H, a chunk that would open on the top rung after H such
+ *      chunks opens one rung lower);
+ *   4. the token is row j of its chunk; rows j < w of a chunk that is not the first of its
+ *      sequence are cross-faded with lambda = (j+1)/(w+1) (Sec. III-D), all others have lambda = 1.
+ * ------------------------------------------------------------------------------------------- */
+int cwlo_stream_reset(cwlo_stream_state* st) {
+  if (!st) return CWLO_ERR_ARG;
+  st->pos = 0; st->len = 0; st->cur_rung = 0; st->prev_rung = -1; st->hi_used = 0; st->first = 1;
+  for (int i = 0; i < CWLO_STREAM_MAX_MIN_LEN; ++i) st->ring[i] = 0;
+  return CWLO_OK;
+}
+
+int cwlo_stream_step(cwlo_stream_state* st, float score, const cwlo_policy* p, cwlo_row_gate* out) {
+  if (!st || !out || !policy_ok(p) || p->min_len > CWLO_STREAM_MAX_MIN_LEN) return CWLO_ERR_ARG;
+  const int32_t L = p->min_len;
+  /* 1. trailing window */
+  st->ring[st->pos % L] = cwlo_quantise(score);
+  const int32_t n_win = (st->pos + 1 < L) ? st->pos + 1 : L;
+  int64_t win = 0;
+  for (int32_t i = 0; i < n_win; ++i) win += st->ring[i];     /* slots 0..n_win-1 hold exactly the last n_win scores */
+  int32_t r_win = cwlo_rung(win, n_win, p);
+  /* 2./3. open a chunk? */
+  int open = 0;
+  if (st->pos == 0) { open = 1; st->first = 1; }
+  else if (st->len >= L && (st->len >= p->max_len || r_win != st->cur_rung)) { open = 1; st->first = 0; }
+  if (open) {
+    if (p->hi_budget >= 0 && p->n_rungs >= 2 && r_win == p->n_rungs - 1) {
+      if (st->hi_used >= p->hi_budget) r_win = p->n_rungs - 2; else st->hi_used += 1;
+    }
+    st->prev_rung = (st->pos == 0) ? -1 : st->cur_rung;
+    st->cur_rung = r_win;
+    st->len = 0;
+  }
+  /* 4. this token's row descriptor */
+  const int32_t j = st->len;
+  st->len += 1;
+  st->pos += 1;
+  out->pos_in_chunk = j;
+  out->opened = open;
+  out->rank_in = p->rung_rank[st->cur_rung];
+  out->scale_in = p->rung_scale[st->cur_rung];
+  out->rank_out = 0; out->scale_out = 0.0f; out->lambda = 1.0f;
+  if (!st->first && j < p->window) {
+    out->lambda = (float)(j + 1) / (float)(p->window + 1);
+    out->rank_out = p->rung_rank[st->prev_rung];
+    out->scale_out = p->rung_scale[st->prev_rung];
+  }
+  return CWLO_OK;
+}
+
+/* Adapted projection with one descriptor per row (decode: every row is another sequence's newest token):
+ *   y_t = x_t W + (1-lam_t) s_out (x_t A[:, :r_out]) B[:r_out, :] + lam_t s_in (x_t A[:, :r_in]) B[:r_in, :]  */
+int cwlo_apply_rows(const uint16_t* X, int64_t ldx, const uint16_t* W, int64_t ldw,
+                    const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
+                    int32_t T, int32_t d_in, int32_t d_out, int32_t R,
+                    const cwlo_row_gate* gates, double* Y, int64_t ldy) {
+  if (!X || !W || !A || !B || !gates || !Y || T < 0 || d_in < 1 || d_out < 1 || R < 1) return CWLO_ERR_ARG;
+  for (int32_t t = 0; t < T; ++t)
+    if (gates[t].rank_in < 0 || gates[t].rank_in > R || gates[t].rank_out < 0 || gates[t].rank_out > R) return CWLO_ERR_ARG;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int32_t t = 0; t < T; ++t) {
+    const uint16_t* x = X + (int64_t)t * ldx;
+    double* y = Y + (int64_t)t * ldy;
+    for (int32_t n = 0; n < d_out; ++n) y[n] = 0.0;
+    for (int32_t k = 0; k < d_in; ++k) {
+      double xk = bf16_to_double(x[k]);
+      const uint16_t* w = W + (int64_t)k * ldw;
+      for (int32_t n = 0; n < d_out; ++n) y[n] += xk * bf16_to_double(w[n]);
+    }
+    double* h = (double*)malloc(sizeof(double) * (size_t)R);
+    double* d_new = (double*)malloc(sizeof(double) * (size_t)d_out);
+    double* d_old = (double*)malloc(sizeof(double) * (size_t)d_out);
+    const double lam = (double)gates[t].lambda;
+    adapter_row(x, A, lda, B, ldb, d_in, d_out, gates[t].rank_in, (double)gates[t].scale_in, h, d_new);
+    if (lam < 1.0) {
+      adapter_row(x, A, lda, B, ldb, d_in, d_out, gates[t].rank_out, (double)gates[t].scale_out, h, d_old);
+      for (int32_t n = 0; n < d_out; ++n) y[n] += (1.0 - lam) * d_old[n] + lam * d_new[n];
+    } else {
+      for (int32_t n = 0; n < d_out; ++n) y[n] += d_new[n];
+    }
+    free(h); free(d_new); free(d_old);
+  }
+  return CWLO_OK;
+}

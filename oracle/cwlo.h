@@ -20,6 +20,8 @@
  *   budget    pinned  (definition: keep the H largest means, earlier index wins ties)
  *   blend     pinned  (weights sum to one, equal spacing, convex combination of single-chunk runs)
  *   apply     pinned  (merged-weight LoRA, r = 0 base, hand-expanded tiny case, linearity)
+ *   stream    parity unpinned against the paper (no rule printed); pinned internally by hand-traced runs,
+ *             invariants and an independent brute force; apply_rows pinned against cwlo_apply on equivalent tables
  */
 #ifndef CWLO_H
 #define CWLO_H
@@ -88,6 +90,31 @@ int cwlo_apply(const uint16_t* X, int64_t ldx, const uint16_t* W, int64_t ldw,
                const int32_t* offsets, const int32_t* rank, const float* scale,
                const int32_t* flags, int32_t n_chunks, int32_t window,
                const int32_t* rows, int32_t n_rows, double* Y, int64_t ldy);
+
+/* Decode-time scheduler state of ONE sequence and the descriptor of one row (see cwlo.c for the rule). */
+#define CWLO_STREAM_MAX_MIN_LEN 64
+typedef struct {
+  int32_t pos;        /* tokens seen */
+  int32_t len;        /* tokens in the open chunk */
+  int32_t cur_rung;   /* rung the open chunk was opened on */
+  int32_t prev_rung;  /* rung of the chunk before it (-1: none) */
+  int32_t hi_used;    /* top-rung chunks opened so far */
+  int32_t first;      /* the open chunk is the first of its sequence */
+  int64_t ring[CWLO_STREAM_MAX_MIN_LEN];  /* quantised scores of the last min_len tokens, slot = position mod min_len */
+} cwlo_stream_state;
+typedef struct {
+  int32_t rank_in, rank_out;      /* prefix ranks of the row's own chunk and of the chunk before it */
+  float   scale_in, scale_out;    /* their gating scales */
+  float   lambda;                 /* cross-fade weight of the own chunk, fp32 (j+1)/(w+1); 1 outside a window */
+  int32_t pos_in_chunk;           /* j */
+  int32_t opened;                 /* 1 if this token opened a chunk */
+} cwlo_row_gate;
+int cwlo_stream_reset(cwlo_stream_state* st);
+int cwlo_stream_step(cwlo_stream_state* st, float score, const cwlo_policy* p, cwlo_row_gate* out);
+int cwlo_apply_rows(const uint16_t* X, int64_t ldx, const uint16_t* W, int64_t ldw,
+                    const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
+                    int32_t T, int32_t d_in, int32_t d_out, int32_t R,
+                    const cwlo_row_gate* gates, double* Y, int64_t ldy);
 
 /* Number of threads the row loops of cwlo_score_tokens / cwlo_apply run on (OpenMP). */
 int  cwlo_get_threads(void);
