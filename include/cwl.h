@@ -149,6 +149,45 @@ cwl_status cwl_apply_grouped(const void* X, int64_t ldx, const cwl_projection* p
                              int32_t T, int32_t d_in, int32_t R, cwl_chunk_table table, int32_t window,
                              void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream);
 
+/* Decode-time scheduler (Sec. III-A "streaming and cached", III-B "grouped online", III-F "state cached across
+ * steps"): every step brings one new token per sequence.  The paper names the constraints only; the rule here is
+ * causal.  Per sequence the state holds the open chunk's length and the rung it was opened on, the rung of the chunk
+ * before it, and the quantised scores of the last min_len tokens.  A new token first enters that trailing window;
+ * the first token of a sequence opens the first chunk on the window's rung; later, a chunk of at least min_len
+ * tokens closes when it holds max_len tokens or when the window's rung differs from the rung it was opened on, and
+ * the token opens a new chunk on the window's rung (one rung lower when that is the top rung and hi_budget such
+ * chunks were opened already).  Rows j < window of a chunk that is not its sequence's first are cross-faded with
+ * lambda = (j+1)/(window+1) (Sec. III-D).  All compares are integer (Q24 sums), so results are bit-exact.
+ *   cwl_stream_state_bytes   size of the DEV state for n_seq sequences (min_len <= CWL_STREAM_MAX_MIN_LEN)
+ *   cwl_stream_reset         all sequences back to "nothing seen"
+ *   cwl_stream_step          score DEV fp32 [n_seq] (the new tokens' complexity scores); active DEV int32 [n_seq] or
+ *                            NULL (0 = this sequence has no token this step: state untouched, its gate has rank 0);
+ *                            gates DEV [n_seq], the row descriptors cwl_apply_rows consumes.  state must be 16-byte aligned.
+ * Errors: INVALID_ARG (NULLs, bad policy, min_len above the limit), WORKSPACE (state missing, small or misaligned). */
+#define CWL_STREAM_MAX_MIN_LEN 64
+typedef struct {
+  int32_t rank_in, rank_out;     /* prefix rank of the row's chunk, and of the chunk before it (used when lambda < 1) */
+  float   scale_in, scale_out;   /* their gating scales */
+  float   lambda;                /* weight of the row's own chunk; 1 outside a cross-fade window */
+  int32_t pos_in_chunk;          /* j; -1 for an inactive sequence */
+  int32_t opened;                /* 1 if this token opened a chunk */
+} cwl_row_gate;
+size_t     cwl_stream_state_bytes(int32_t n_seq, int32_t min_len);
+cwl_status cwl_stream_reset(void* state, size_t state_bytes, int32_t n_seq, int32_t min_len, void* stream);
+cwl_status cwl_stream_step(const float* score, const int32_t* active, int32_t n_seq, const cwl_policy* policy,
+                           void* state, size_t state_bytes, cwl_row_gate* gates, void* stream);
+
+/* cwl_apply with one descriptor per row instead of a chunk table (decode: every row is another sequence's newest
+ * token, so rows inside a cross-fade window are blended too):
+ *   y_t = x_t W + (1 - lambda_t) scale_out_t (x_t A[:, :rank_out_t]) B[:rank_out_t, :]
+ *               + lambda_t scale_in_t (x_t A[:, :rank_in_t]) B[:rank_in_t, :]
+ * gates DEV [T]; ranks are clamped to [0, R].  Everything else as cwl_apply (same workspace size). */
+cwl_status cwl_apply_rows(const void* X, int64_t ldx, const void* W, int64_t ldw,
+                          const void* A, int64_t lda, const void* B, int64_t ldb,
+                          int32_t T, int32_t d_in, int32_t d_out, int32_t R,
+                          const cwl_row_gate* gates, void* Y, int64_t ldy,
+                          void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream);
+
 /* The schedule cwl_apply uses for a shape when `pairs` CTA pairs can be resident (a B200 holds 74): how
  * the output is cut into column tiles (Sec. III-F leaves the kernel schedule open; this is the library's own
  * design), whether the K loop of decode-sized problems is split, and who computes the shrink X A.

@@ -21,7 +21,8 @@ STATUS = {0: "CWL_OK", 1: "CWL_ERR_INVALID_ARG", 2: "CWL_ERR_SHAPE", 3: "CWL_ERR
 
 EXPORTS = ["cwl_status_string", "cwl_version", "cwl_score_tokens", "cwl_partition_workspace_bytes",
            "cwl_partition", "cwl_apply_workspace_bytes", "cwl_apply", "cwl_apply_grouped_workspace_bytes",
-           "cwl_apply_grouped", "cwl_apply_plan",
+           "cwl_apply_grouped", "cwl_apply_plan", "cwl_stream_state_bytes", "cwl_stream_reset", "cwl_stream_step",
+           "cwl_apply_rows",
            "cwl_apply_noalloc_scratch_need", "cwl_apply_noalloc"]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 
@@ -48,6 +49,15 @@ class CChunkTable(C.Structure):
 
 
 MAX_GROUP = 4
+STREAM_MAX_MIN_LEN = 64
+
+
+class CRowGate(C.Structure):
+    _fields_ = [("rank_in", C.c_int32), ("rank_out", C.c_int32), ("scale_in", C.c_float), ("scale_out", C.c_float),
+                ("lam", C.c_float), ("pos_in_chunk", C.c_int32), ("opened", C.c_int32)]
+
+
+ROW_GATE_BYTES = C.sizeof(CRowGate)     # 28: gates live in a uint8 tensor of [n, ROW_GATE_BYTES]
 
 
 class CProjection(C.Structure):
@@ -95,6 +105,17 @@ def lib():
         L.cwl_apply_grouped.restype = C.c_int
         L.cwl_apply_grouped.argtypes = [C.c_void_p, C.c_int64, C.POINTER(CProjection), C.c_int32, C.c_int32, C.c_int32,
                                         C.c_int32, CChunkTable, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        L.cwl_stream_state_bytes.restype = C.c_size_t
+        L.cwl_stream_state_bytes.argtypes = [C.c_int32, C.c_int32]
+        L.cwl_stream_reset.restype = C.c_int
+        L.cwl_stream_reset.argtypes = [C.c_void_p, C.c_size_t, C.c_int32, C.c_int32, C.c_void_p]
+        L.cwl_stream_step.restype = C.c_int
+        L.cwl_stream_step.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(CPolicy), C.c_void_p, C.c_size_t,
+                                      C.c_void_p, C.c_void_p]
+        L.cwl_apply_rows.restype = C.c_int
+        L.cwl_apply_rows.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
+                                     C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                     C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         L.cwl_apply_plan.restype = C.c_int
         L.cwl_apply_plan.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(CApplyPlanInfo)]
         L.cwl_apply_noalloc_scratch_need.restype = C.c_size_t
@@ -277,6 +298,59 @@ def cwl_apply_grouped(X: torch.Tensor, Ws: Sequence[torch.Tensor], As: Optional[
                                                         _p(workspace), workspace.numel(), _p(status_word),
                                                         _stream_ptr(stream)))
     return Ys
+
+
+def cwl_stream_state_bytes(n_seq: int, min_len: int) -> int:
+    return int(lib().cwl_stream_state_bytes(n_seq, min_len))
+
+
+class DeviceStream:
+    """Device-resident decode-time scheduler state of n_seq sequences plus the row-gate buffer it fills."""
+
+    def __init__(self, n_seq: int, policy: CPolicy, device="cuda"):
+        self.n_seq, self.policy = int(n_seq), policy
+        self.state = torch.empty(max(cwl_stream_state_bytes(n_seq, int(policy.min_len)), 16), dtype=torch.uint8, device=device)
+        self.gates = torch.zeros(max(n_seq, 1), ROW_GATE_BYTES, dtype=torch.uint8, device=device)
+        self.reset()
+
+    def reset(self, stream: Optional[torch.cuda.Stream] = None) -> None:
+        _check("cwl_stream_reset", lib().cwl_stream_reset(_p(self.state), self.state.numel(), self.n_seq,
+                                                          int(self.policy.min_len), _stream_ptr(stream)))
+
+    def step(self, score: torch.Tensor, active: Optional[torch.Tensor] = None,
+             stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """Advances every (active) sequence by one token; returns the gate buffer ([n_seq, 28] bytes on the device)."""
+        assert score.is_cuda and score.dtype == torch.float32 and score.is_contiguous() and score.numel() == self.n_seq
+        if active is not None:
+            assert active.is_cuda and active.dtype == torch.int32 and active.is_contiguous()
+        _check("cwl_stream_step", lib().cwl_stream_step(_p(score), _p(active), self.n_seq, C.byref(self.policy),
+                                                        _p(self.state), self.state.numel(), _p(self.gates),
+                                                        _stream_ptr(stream)))
+        return self.gates
+
+    def gates_to_host(self):
+        import numpy as np
+        dt = np.dtype([("rank_in", np.int32), ("rank_out", np.int32), ("scale_in", np.float32), ("scale_out", np.float32),
+                       ("lam", np.float32), ("pos_in_chunk", np.int32), ("opened", np.int32)])
+        return self.gates[:self.n_seq].cpu().numpy().view(dt).reshape(self.n_seq)
+
+
+def cwl_apply_rows(X: torch.Tensor, W: torch.Tensor, A: torch.Tensor, B: torch.Tensor, gates: torch.Tensor,
+                   Y: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                   status_word: Optional[torch.Tensor] = None,
+                   stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """cwl_apply with one (rank, scale, lambda) descriptor per row; ``gates`` is a [T, 28]-byte device tensor."""
+    T, d_in = X.shape
+    d_out, R = W.shape[1], A.shape[1]
+    assert gates.is_cuda and gates.dtype == torch.uint8 and gates.is_contiguous() and gates.numel() >= T * ROW_GATE_BYTES
+    if Y is None:
+        Y = torch.empty(T, d_out, dtype=torch.bfloat16, device=X.device)
+    if workspace is None:
+        workspace = torch.empty(cwl_apply_workspace_bytes(T, d_in, d_out, R), dtype=torch.uint8, device=X.device)
+    _check("cwl_apply_rows", lib().cwl_apply_rows(_p(X), X.stride(0), _p(W), W.stride(0), _p(A), A.stride(0),
+                                                  _p(B), B.stride(0), T, d_in, d_out, R, _p(gates), _p(Y), Y.stride(0),
+                                                  _p(workspace), workspace.numel(), _p(status_word), _stream_ptr(stream)))
+    return Y
 
 
 def cwl_apply_noalloc(X: torch.Tensor, W: torch.Tensor, A: Optional[torch.Tensor], B: Optional[torch.Tensor],

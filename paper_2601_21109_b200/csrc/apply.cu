@@ -100,6 +100,7 @@ struct ApplyParams {
   int* flags;              // [2 n_m_pairs] 1 once H' of the 128-row tile is published
   int* sk_counters;        // [2 tiles] split-K partials stored per (tile, CTA rank)
   cwl_chunk_table table;
+  const cwl_row_gate* row_gates;   // when set: one descriptor per row instead of the chunk table
   int32_t* status_word;
   Plan plan;
 };
@@ -335,6 +336,18 @@ __device__ __forceinline__ bool get_item(int i, int b, int sh_begin, const Apply
 // Per-row gate from the chunk table (Sec. III-C rank mask and scale, Sec. III-D cross-fade weight).
 __device__ __forceinline__ RowGate row_gate(int t, const ApplyParams& p) {
   RowGate g{0.f, 0.f, 0, 0};
+  if (p.row_gates != nullptr) {
+    if (t < p.T) {
+      const cwl_row_gate d = p.row_gates[t];
+      g.r_in = min(max(d.rank_in, 0), p.R);
+      g.w_in = d.lambda * d.scale_in;
+      if (d.lambda < 1.f) {
+        g.r_out = min(max(d.rank_out, 0), p.R);
+        g.w_out = (1.f - d.lambda) * d.scale_out;
+      }
+    }
+    return g;
+  }
   const cwl_chunk_table& tb = p.table;
   const int C = min(*tb.n_chunks, tb.capacity);
   if (t < p.T && C > 0 && t >= tb.offsets[0] && t < tb.offsets[C]) {
@@ -1105,7 +1118,7 @@ size_t carve_apply(ApplyWorkspace& w, char* base, const Plan& pl, int T, int R) 
 
 // Argument checks shared by every entry point.  `adapter` comes back true when every projection has both factors.
 cwl_status check_group(const void* X, int64_t ldx, const cwl_projection* proj, int n_proj, int T, int d_in, int R,
-                       const cwl_chunk_table& table, int window, bool& adapter) {
+                       const cwl_chunk_table& table, const cwl_row_gate* row_gates, int window, bool& adapter) {
   if (proj == nullptr || n_proj < 1 || n_proj > CWL_MAX_GROUP) return CWL_ERR_INVALID_ARG;
   if (T < 0 || d_in < 1 || R < 0 || window < 0) return CWL_ERR_INVALID_ARG;
   if (T > 0 && X == nullptr) return CWL_ERR_INVALID_ARG;
@@ -1126,8 +1139,9 @@ cwl_status check_group(const void* X, int64_t ldx, const cwl_projection* proj, i
     if (q.ldw % 8 != 0 || q.ldy % 8 != 0 || (adapter && (q.lda % 8 != 0 || q.ldb % 8 != 0))) return CWL_ERR_SHAPE;
     if (!aligned16(q.W) || !aligned16(q.Y) || (adapter && (!aligned16(q.A) || !aligned16(q.B)))) return CWL_ERR_SHAPE;
   }
-  if (adapter && (table.offsets == nullptr || table.rank == nullptr || table.scale == nullptr ||
-                  table.flags == nullptr || table.n_chunks == nullptr || table.capacity < 0))
+  if (adapter && row_gates == nullptr &&
+      (table.offsets == nullptr || table.rank == nullptr || table.scale == nullptr ||
+       table.flags == nullptr || table.n_chunks == nullptr || table.capacity < 0))
     return CWL_ERR_INVALID_ARG;
   return CWL_OK;
 }
@@ -1136,9 +1150,9 @@ cwl_status check_group(const void* X, int64_t ldx, const cwl_projection* proj, i
 cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* proj, int n_proj, int32_t T,
                             int32_t d_in, int32_t R, cwl_chunk_table table, int32_t window, void* workspace,
                             size_t workspace_bytes, int32_t* status_word, void* stream_, bool allow_split_k,
-                            size_t scratch_limit) {
+                            size_t scratch_limit, const cwl_row_gate* row_gates = nullptr) {
   bool adapter = false;
-  const cwl_status chk = check_group(X, ldx, proj, n_proj, T, d_in, R, table, window, adapter);
+  const cwl_status chk = check_group(X, ldx, proj, n_proj, T, d_in, R, table, row_gates, window, adapter);
   if (chk != CWL_OK) return chk;
   if (T == 0) return CWL_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -1179,7 +1193,7 @@ cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* pr
   for (int j = 0; j < n_proj; ++j) { p.Y[j] = static_cast<__nv_bfloat16*>(proj[j].Y); p.ldy[j] = proj[j].ldy; }
   p.Hg = ws.Hg; p.partial = ws.partial; p.sk_partial = ws.sk_partial;
   p.counters = ws.sync; p.flags = ws.sync + 2 * pl.n_m_pairs; p.sk_counters = ws.sync + 4 * pl.n_m_pairs;
-  p.table = table; p.status_word = status_word;
+  p.table = table; p.row_gates = row_gates; p.status_word = status_word;
   p.plan = pl;
 
   // the counters and flags are the only words that must start at zero
@@ -1263,6 +1277,20 @@ extern "C" cwl_status cwl_apply_grouped(const void* X, int64_t ldx, const cwl_pr
                                         void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream) {
   return cwl::apply_group_impl(X, ldx, proj, n_proj, T, d_in, R, table, window, workspace, workspace_bytes,
                                status_word, stream, true, 0);
+}
+
+extern "C" cwl_status cwl_apply_rows(const void* X, int64_t ldx, const void* W, int64_t ldw,
+                                     const void* A, int64_t lda, const void* B, int64_t ldb,
+                                     int32_t T, int32_t d_in, int32_t d_out, int32_t R,
+                                     const cwl_row_gate* gates, void* Y, int64_t ldy,
+                                     void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream) {
+  if (gates == nullptr || A == nullptr || B == nullptr || R < 1) return CWL_ERR_INVALID_ARG;
+  cwl_projection q;
+  q.W = W; q.ldw = ldw; q.A = A; q.lda = lda; q.B = B; q.ldb = ldb; q.Y = Y; q.ldy = ldy; q.d_out = d_out;
+  cwl_chunk_table none;
+  memset(&none, 0, sizeof(none));
+  return cwl::apply_group_impl(X, ldx, &q, 1, T, d_in, R, none, 0, workspace, workspace_bytes, status_word, stream,
+                               true, 0, gates);
 }
 
 // ------------------------------------------------------------------------------ no-allocation variant
