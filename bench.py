@@ -137,8 +137,15 @@ def make_workload(name: str):
         return wl.config2()
     if name == "cfg1":
         return wl.config1()
-    if name == "cfg4":
-        return wl.config4()
+    if name in ("cfg4", "cfg4_stream"):
+        w = wl.config4()
+        if name == "cfg4_stream":
+            # decode through the token-by-token scheduler: per-sequence scores U[0,1) stand in for the scorer's output
+            from paper_2601_21109_b200.workloads import Policy
+            w.name = "cfg4_decode_streaming_scheduler"
+            w.policy = Policy.ladder([8, 16, 32, 64], 32.0, [0.25, 0.5, 0.75], min_len=16, window=8)
+            w.score = np.random.default_rng(wl.SEED_BASE + 4).uniform(0, 1, w.T).astype(np.float32)
+        return w
     if name == "cfg3":
         return wl.config3()
     if name == "cfg5":
@@ -237,7 +244,8 @@ def run_ours(args):
 
     w = make_workload(args.workload)
     n_layers = args.layers if args.workload == "cfg5" else 1
-    hp = HotPath(w, n_layers=n_layers, grouped=not args.no_group)
+    streaming = args.workload == "cfg4_stream"
+    hp = HotPath(w, n_layers=n_layers, grouped=not args.no_group, streaming=streaming)
     stream = torch.cuda.current_stream()
 
     # thresholds of the rule-based percentile mapping (Sec. IV-C): quartiles of this batch's scores
@@ -273,6 +281,8 @@ def run_ours(args):
     t_wall0 = time.time()
     e0.record(stream)
     for i in range(args.steps):
+        if streaming:
+            hp.stream_state.step(hp.score)
         for layer in range(n_layers):
             if hp.logits is not None:
                 hp.score_step()
@@ -360,7 +370,7 @@ def run_ours(args):
     peaks = load_peaks()
     apply_avg_ms = float(np.mean(apply_ms))
     region_s = ms_total * 1e-3
-    if args.workload == "cfg4":
+    if args.workload in ("cfg4", "cfg4_stream"):
         bytes_alg = sum(2 * (hp.T * di + di * do + hp.R * (di + do) + hp.T * do) + 2 * hp.T * hp.R * 2 for di, do in proj_dims)
         achieved = bytes_alg / (apply_avg_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -384,7 +394,7 @@ def run_ours(args):
     roof["executed_tflops"] = f_exe / (apply_avg_ms * 1e-3) / 1e12
     roof["frac_of_nominal_2250"] = (f_alg / (apply_avg_ms * 1e-3) / 1e12) / 2250.0
 
-    parts = (["score"] if hp.logits is not None else []) + ([] if hp.fixed_table else ["partition"]) + \
+    parts = (["scheduler step"] if streaming else []) + (["score"] if hp.logits is not None else []) + ([] if hp.fixed_table else ["partition"]) + \
         [f"{len(hp.projs)} projections in {len(hp.launch_groups())} apply launches"]
     steps_include = (f"{n_layers} layers x (" if n_layers > 1 else "(") + " + ".join(parts) + ")"
     step_bytes = n_layers * (sum(2 * p.d_in * p.d_out for p in hp.projs) +
@@ -429,7 +439,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg4_stream", "cfg5"])
     ap.add_argument("--layers", type=int, default=32, help="layers of the cfg5 projection stack (a step runs all of them)")
     ap.add_argument("--no-group", action="store_true",
                     help="one cwl_apply launch per projection instead of grouped launches for q,k,v and gate,up")

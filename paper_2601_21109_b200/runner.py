@@ -36,8 +36,11 @@ class HotPath:
     """Device-resident state of one layer's adapted projections plus the scheduler in front."""
 
     def __init__(self, w: Workload, device: str = "cuda", keep_host: bool = False, n_layers: int = 1,
-                 grouped: bool = True):
+                 grouped: bool = True, streaming: bool = False):
         self.grouped = grouped
+        # decode with the token-by-token scheduler: every step the cached per-sequence state advances by one
+        # token (the rows' scores) and the projections take the row gates it emits instead of a chunk table
+        self.streaming = streaming
         self.T, self.R, self.policy = w.T, w.R, w.policy
         self.device = device
         self.cu_seqlens = torch.from_numpy(w.cu_seqlens).to(device)
@@ -73,6 +76,7 @@ class HotPath:
         self.apply_ws = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
         self.cpolicy = policy_struct(w.policy)
+        self.stream_state = cwl.DeviceStream(w.T, self.cpolicy, device) if streaming else None
 
     # launches per call, for the benchmark's kernel count
     LAUNCHES_SCORE = 1
@@ -112,6 +116,11 @@ class HotPath:
         return out
 
     def apply_step(self, table: Optional[cwl.DeviceChunkTable] = None, dense: bool = False, layer: int = 0) -> None:
+        if self.streaming and table is None and not dense:
+            for p in self.layers[layer]:
+                cwl.cwl_apply_rows(self.X[p.d_in], p.W, p.A, p.B, self.stream_state.gates, Y=p.Y,
+                                   workspace=self.apply_ws, status_word=self.status)
+            return
         tab = table if table is not None else self.table
         for group in self.launch_groups(layer):
             p = group[0]
@@ -125,6 +134,8 @@ class HotPath:
 
     def step(self) -> None:
         """One pass of the whole hot path on the current stream (no host synchronisation)."""
+        if self.streaming:
+            self.stream_state.step(self.score)
         for layer in range(len(self.layers)):
             if self.logits is not None:
                 self.score_step()
@@ -138,4 +149,4 @@ class HotPath:
             n += self.LAUNCHES_SCORE
         if not self.fixed_table:
             n += self.LAUNCHES_PARTITION
-        return n * len(self.layers)
+        return n * len(self.layers) + (1 if self.streaming else 0)
