@@ -228,18 +228,15 @@ def run_reference(args):
 # ---------------------------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
-    import torch.distributed as dist
     from paper_2601_21109_b200 import binding as cwl
     from paper_2601_21109_b200.runner import HotPath
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2601_21109_b200 import replicas
+    rank, local_rank, world = replicas.world_from_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    replicas.init("nccl", local_rank, world)
     cwl.lib()  # fails loudly when libcwl.so is missing
 
     w = make_workload(args.workload)
@@ -263,9 +260,7 @@ def run_ours(args):
     f_alg, f_exe = f_alg * n_layers, f_exe * n_layers
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        replicas.barrier(world)
 
     # ---- device-resident timing --------------------------------------------------------------
     for _ in range(args.warmup):
@@ -297,14 +292,10 @@ def run_ours(args):
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     ms_total = e0.elapsed_time(e1)
     apply_ms = [sum(a.elapsed_time(b) for a, b in ev[i * n_layers:(i + 1) * n_layers]) for i in range(args.steps)]
-    if world > 1:
-        t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = replicas.max_over_ranks(ms_total, world)
     if int(hp.status.item()) != 0:
         raise SystemExit(f"device status word {int(hp.status.item()):#x}")
-    tokens_total = hp.T * args.steps * world
-    value = tokens_total / (ms_total * 1e-3)
+    value = replicas.job_throughput(hp.T, args.steps, world, ms_total)
 
     # ---- comparison runs through the same kernels: static full-rank LoRA and the dense floor ---
     from paper_2601_21109_b200 import workloads as wl
@@ -355,15 +346,11 @@ def run_ours(args):
         b.record(stream)
         barrier()
         e2e_ms = a.elapsed_time(b)
-        if world > 1:
-            t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        e2e_value = hp.T * e2e_steps * world / (e2e_ms * 1e-3)
+        e2e_ms = replicas.max_over_ranks(e2e_ms, world)
+        e2e_value = replicas.job_throughput(hp.T, e2e_steps, world, e2e_ms)
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        replicas.finish(world)
         return
 
     # ---- roofline of the dominant kernel (the projection GEMM inside cwl_apply) -----------------
@@ -429,8 +416,7 @@ def run_ours(args):
         "cpu_baseline": dict(value=cpu_val, unit=UNIT, **cpu_info),
     }
     print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.finish(world)
 
 
 def main():
