@@ -254,3 +254,25 @@ def apply_rows(X: np.ndarray, W: np.ndarray, A: np.ndarray, B: np.ndarray, gates
     if rc != 0:
         raise ValueError(f"cwlo_apply_rows: status {rc}")
     return Y
+
+
+# ------------------------------------------------------------------ further complexity signals (Sec. III-A (ii), (iv))
+class _SignalMix(C.Structure):
+    _fields_ = [("w_entropy", C.c_float), ("w_novelty", C.c_float), ("w_prior", C.c_float),
+                ("ngram", C.c_int32), ("context", C.c_int32), ("prior_span", C.c_int32)]
+
+
+def score_tokens_mixed(logits: np.ndarray, token_ids: np.ndarray, cu_seqlens: np.ndarray, w_entropy: float,
+                       w_novelty: float, w_prior: float, ngram: int, context: int, prior_span: int) -> np.ndarray:
+    """clamp(w_e * entropy + w_n * n-gram novelty + w_p * positional prior, 0, 1) per token, fp64 [T]."""
+    z = np.ascontiguousarray(logits, dtype=np.float32)
+    ids = np.ascontiguousarray(token_ids, dtype=np.int32)
+    cu = np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+    T, V = z.shape
+    mix = _SignalMix(float(w_entropy), float(w_novelty), float(w_prior), int(ngram), int(context), int(prior_span))
+    out = np.empty(T, dtype=np.float64)
+    rc = lib().cwlo_score_tokens_mixed(_ptr(z), C.c_int64(V), C.c_int32(T), C.c_int32(V), _ptr(ids), _ptr(cu),
+                                       C.c_int32(len(cu) - 1), C.byref(mix), _ptr(out))
+    if rc != 0:
+        raise ValueError(f"cwlo_score_tokens_mixed: status {rc}")
+    return out

@@ -373,3 +373,47 @@ int cwlo_apply_rows(const uint16_t* X, int64_t ldx, const uint16_t* W, int64_t l
   }
   return CWLO_OK;
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * Token complexity estimator with the further signals of Sec. III-A: (i) next-token entropy,
+ * (ii) n-gram novelty against the recent context, (iv) a positional prior that favours early
+ * steps.  The paper lists the signals and gives no formula; this build's reading:
+ *   e_t   normalised entropy of the token's logit row (as cwlo_score_tokens)
+ *   nu_t  1 if the n-gram ending at t (token ids x[t-n+1..t]) ends at none of the previous
+ *         `context` positions of the same sequence, else 0; the first n-1 tokens of a sequence,
+ *         which have no complete n-gram yet, count as novel
+ *   pi_t  max(0, 1 - p / prior_span), p = position of t inside its sequence
+ *   score = clamp(w_e e_t + w_n nu_t + w_p pi_t, 0, 1)      (a NaN entropy stays NaN)
+ * ------------------------------------------------------------------------------------------- */
+int cwlo_score_tokens_mixed(const float* logits, int64_t ld, int32_t T, int32_t V,
+                            const int32_t* token_ids, const int32_t* cu, int32_t n_seq,
+                            const cwlo_signal_mix* mix, double* score) {
+  if (!logits || !token_ids || !cu || !mix || !score || T < 0 || V < 2 || ld < V || n_seq < 0) return CWLO_ERR_ARG;
+  if (mix->ngram < 1 || mix->ngram > 8 || mix->context < 1 || mix->prior_span < 1) return CWLO_ERR_ARG;
+  if (!(mix->w_entropy >= 0.f) || !(mix->w_novelty >= 0.f) || !(mix->w_prior >= 0.f)) return CWLO_ERR_ARG;
+  if (cu[0] != 0 || cu[n_seq] != T) return CWLO_ERR_ARG;
+  for (int32_t s = 0; s < n_seq; ++s) {
+    if (cu[s + 1] < cu[s]) return CWLO_ERR_ARG;
+    for (int32_t t = cu[s]; t < cu[s + 1]; ++t) {
+      const int32_t p = t - cu[s];
+      const double e = entropy_row(logits + (int64_t)t * ld, V);
+      double nu = 1.0;
+      if (p >= mix->ngram - 1) {
+        int32_t lo = t - mix->context;
+        if (lo < cu[s] + mix->ngram - 1) lo = cu[s] + mix->ngram - 1;
+        for (int32_t u = lo; u < t && nu == 1.0; ++u) {
+          int same = 1;
+          for (int32_t i = 0; i < mix->ngram; ++i)
+            if (token_ids[u - i] != token_ids[t - i]) { same = 0; break; }
+          if (same) nu = 0.0;
+        }
+      }
+      double pi = 1.0 - (double)p / (double)mix->prior_span;
+      if (pi < 0.0) pi = 0.0;
+      double v = (double)mix->w_entropy * e + (double)mix->w_novelty * nu + (double)mix->w_prior * pi;
+      if (!isnan(v)) { if (v < 0.0) v = 0.0; if (v > 1.0) v = 1.0; }
+      score[t] = v;
+    }
+  }
+  return CWLO_OK;
+}

@@ -20,6 +20,7 @@
  *   budget    pinned  (definition: keep the H largest means, earlier index wins ties)
  *   blend     pinned  (weights sum to one, equal spacing, convex combination of single-chunk runs)
  *   apply     pinned  (merged-weight LoRA, r = 0 base, hand-expanded tiny case, linearity)
+ *   mixed     pinned  (weights (1,0,0) = entropy score, hand-traced novelty, closed-form prior, set-based brute force)
  *   stream    parity unpinned against the paper (no rule printed); pinned internally by hand-traced runs,
  *             invariants and an independent brute force; apply_rows pinned against cwlo_apply on equivalent tables
  */
@@ -90,6 +91,17 @@ int cwlo_apply(const uint16_t* X, int64_t ldx, const uint16_t* W, int64_t ldw,
                const int32_t* offsets, const int32_t* rank, const float* scale,
                const int32_t* flags, int32_t n_chunks, int32_t window,
                const int32_t* rows, int32_t n_rows, double* Y, int64_t ldy);
+
+/* Mix of complexity signals (Sec. III-A (i), (ii), (iv)); see cwlo.c for the definitions. */
+typedef struct {
+  float   w_entropy, w_novelty, w_prior;   /* non-negative weights */
+  int32_t ngram;                           /* n of the n-gram, 1..8 */
+  int32_t context;                         /* previous positions searched, >= 1 */
+  int32_t prior_span;                      /* positions over which the prior falls from 1 to 0, >= 1 */
+} cwlo_signal_mix;
+int cwlo_score_tokens_mixed(const float* logits, int64_t ld, int32_t T, int32_t V,
+                            const int32_t* token_ids, const int32_t* cu_seqlens, int32_t n_seq,
+                            const cwlo_signal_mix* mix, double* score);
 
 /* Decode-time scheduler state of ONE sequence and the descriptor of one row (see cwlo.c for the rule). */
 #define CWLO_STREAM_MAX_MIN_LEN 64
