@@ -80,6 +80,23 @@ int         cwl_version(void);
 cwl_status cwl_score_tokens(const float* logits, int64_t ld_logits, int32_t T, int32_t V,
                             float* score, void* stream);
 
+/* The estimator with the further signals of Sec. III-A mixed in (the paper lists them without formulas):
+ *   e_t   the entropy score above
+ *   nu_t  n-gram novelty: 1 if the n-gram of token ids ending at t ends at none of the previous `context`
+ *         positions of the same sequence, else 0 (the first n-1 tokens of a sequence count as novel)
+ *   pi_t  positional prior max(0, 1 - p / prior_span), p = position inside the sequence
+ *   score[t] = clamp(w_entropy e_t + w_novelty nu_t + w_prior pi_t, 0, 1);  a NaN e_t stays NaN.
+ * One pass, one kernel: the n-gram search runs in the block that reduces the row.
+ *   token_ids DEV int32 [T]; cu_seqlens DEV int32 [n_seq + 1] (cu[0] = 0, cu[n_seq] = T, unchecked on device)
+ * Errors: INVALID_ARG (NULLs, negative weight, ngram outside 1..8, context or prior_span < 1), SHAPE. */
+typedef struct {
+  float   w_entropy, w_novelty, w_prior;
+  int32_t ngram, context, prior_span;
+} cwl_signal_mix;
+cwl_status cwl_score_tokens_mixed(const float* logits, int64_t ld_logits, int32_t T, int32_t V,
+                                  const int32_t* token_ids, const int32_t* cu_seqlens, int32_t n_seq,
+                                  const cwl_signal_mix* mix, float* score, void* stream);
+
 /* Adaptive chunker and rank-ladder selector (Sec. III-B, III-C).
  * Scores are quantised to q = floor(clamp(s,0,1) * 2^24) (NaN -> 2^24) and every mean is compared
  * as an integer sum, so the result depends on the fp32 score array only.  Per sequence a greedy

@@ -19,7 +19,7 @@ MAX_RUNGS = 8
 STATUS = {0: "CWL_OK", 1: "CWL_ERR_INVALID_ARG", 2: "CWL_ERR_SHAPE", 3: "CWL_ERR_UNSUPPORTED",
           4: "CWL_ERR_CAPACITY", 5: "CWL_ERR_WORKSPACE", 6: "CWL_ERR_CUDA", 7: "CWL_ERR_TIMEOUT"}
 
-EXPORTS = ["cwl_status_string", "cwl_version", "cwl_score_tokens", "cwl_partition_workspace_bytes",
+EXPORTS = ["cwl_status_string", "cwl_version", "cwl_score_tokens", "cwl_score_tokens_mixed", "cwl_partition_workspace_bytes",
            "cwl_partition", "cwl_apply_workspace_bytes", "cwl_apply", "cwl_apply_grouped_workspace_bytes",
            "cwl_apply_grouped", "cwl_apply_plan", "cwl_stream_state_bytes", "cwl_stream_reset", "cwl_stream_step",
            "cwl_apply_rows",
@@ -65,6 +65,11 @@ class CProjection(C.Structure):
                 ("B", C.c_void_p), ("ldb", C.c_int64), ("Y", C.c_void_p), ("ldy", C.c_int64), ("d_out", C.c_int32)]
 
 
+class CSignalMix(C.Structure):
+    _fields_ = [("w_entropy", C.c_float), ("w_novelty", C.c_float), ("w_prior", C.c_float),
+                ("ngram", C.c_int32), ("context", C.c_int32), ("prior_span", C.c_int32)]
+
+
 class CApplyPlanInfo(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "pairs", "row_tiles", "wide_width", "wide_tiles_per_row", "narrow_width", "narrow_tiles_per_row",
@@ -88,6 +93,9 @@ def lib():
         L.cwl_version.restype = C.c_int
         L.cwl_score_tokens.restype = C.c_int
         L.cwl_score_tokens.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        L.cwl_score_tokens_mixed.restype = C.c_int
+        L.cwl_score_tokens_mixed.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                             C.c_int32, C.POINTER(CSignalMix), C.c_void_p, C.c_void_p]
         L.cwl_partition_workspace_bytes.restype = C.c_size_t
         L.cwl_partition_workspace_bytes.argtypes = [C.c_int32, C.c_int32]
         L.cwl_partition.restype = C.c_int
@@ -202,6 +210,24 @@ def cwl_score_tokens(logits: torch.Tensor, score: Optional[torch.Tensor] = None,
         score = torch.empty(T, dtype=torch.float32, device=logits.device)
     _check("cwl_score_tokens", lib().cwl_score_tokens(_p(logits), logits.stride(0) if T > 1 else max(V, logits.stride(0)),
                                                       T, V, _p(score), _stream_ptr(stream)))
+    return score
+
+
+def cwl_score_tokens_mixed(logits: torch.Tensor, token_ids: torch.Tensor, cu_seqlens: torch.Tensor,
+                           w_entropy: float, w_novelty: float, w_prior: float, ngram: int, context: int,
+                           prior_span: int, score: Optional[torch.Tensor] = None,
+                           stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Entropy, n-gram novelty and positional prior mixed into one score per token (one kernel)."""
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.dim() == 2 and logits.stride(1) == 1
+    assert token_ids.is_cuda and token_ids.dtype == torch.int32 and token_ids.is_contiguous()
+    assert cu_seqlens.is_cuda and cu_seqlens.dtype == torch.int32 and cu_seqlens.is_contiguous()
+    T, V = logits.shape
+    if score is None:
+        score = torch.empty(T, dtype=torch.float32, device=logits.device)
+    mix = CSignalMix(float(w_entropy), float(w_novelty), float(w_prior), int(ngram), int(context), int(prior_span))
+    _check("cwl_score_tokens_mixed", lib().cwl_score_tokens_mixed(
+        _p(logits), logits.stride(0) if T > 1 else max(V, logits.stride(0)), T, V, _p(token_ids), _p(cu_seqlens),
+        cu_seqlens.numel() - 1, C.byref(mix), _p(score), _stream_ptr(stream)))
     return score
 
 

@@ -53,15 +53,54 @@ __device__ __forceinline__ Triple merge(Triple a, Triple b) {
   return a;
 }
 
+// Further signals of Sec. III-A mixed into the score (kMixed): (ii) n-gram novelty against the previous
+// `context` positions of the same sequence, (iv) a positional prior max(0, 1 - p / prior_span).
+struct MixParams {
+  const int32_t* token_ids;   // [T]
+  const int32_t* cu_seqlens;  // [n_seq + 1]
+  int n_seq;
+  float w_entropy, w_novelty, w_prior;
+  int ngram, context, prior_span;
+};
+
+template <bool kMixed>
 __global__ void __launch_bounds__(kScoreThreads)
-score_rows_kernel(const float* __restrict__ logits, int64_t ld, int T, int V, float* __restrict__ score) {
+score_rows_kernel(const float* __restrict__ logits, int64_t ld, int T, int V, float* __restrict__ score,
+                  const MixParams mp) {
   __shared__ Triple warp_part[kScoreThreads / 32];
   __shared__ int warp_bad[kScoreThreads / 32];
+  __shared__ int seq_start;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const float inv_ln_v = 1.0f / logf((float)V);
 
   for (int row = blockIdx.x; row < T; row += gridDim.x) {
     const float* z = logits + (int64_t)row * ld;
+    int novel = 1, p_in_seq = 0;
+    if (kMixed) {
+      // the row's sequence (binary search by one thread), then every thread compares the n-gram ending at this
+      // token with the n-grams ending at its share of the previous `context` positions
+      if (tid == 0) {
+        int lo = 0, hi = mp.n_seq;                   // cu[lo] <= row < cu[hi]
+        while (hi - lo > 1) {
+          const int mid = (lo + hi) >> 1;
+          if (mp.cu_seqlens[mid] <= row) lo = mid; else hi = mid;
+        }
+        seq_start = mp.cu_seqlens[lo];
+      }
+      __syncthreads();
+      const int start = seq_start;
+      p_in_seq = row - start;
+      int found = 0;
+      if (p_in_seq >= mp.ngram - 1) {
+        const int lo = max(row - mp.context, start + mp.ngram - 1);
+        for (int u = row - 1 - tid; u >= lo; u -= kScoreThreads) {
+          bool same = true;
+          for (int i = 0; i < mp.ngram; ++i) same = same && (mp.token_ids[u - i] == mp.token_ids[row - i]);
+          found |= same ? 1 : 0;
+        }
+      }
+      novel = __syncthreads_or(found) ? 0 : 1;
+    }
     Triple acc{-CUDART_INF_F, 0.f, 0.f};
     bool ok = true;  // stays true while every logit is finite or -inf
 
@@ -129,6 +168,11 @@ score_rows_kernel(const float* __restrict__ logits, int64_t ld, int T, int V, fl
           // H = ln S - (U ln2) / S  with U in the log2 domain
           float H = logf(a.S) - (a.U * kLn2) / a.S;
           s = fminf(fmaxf(H * inv_ln_v, 0.f), 1.f);
+          if (kMixed) {
+            const float prior = fmaxf(0.f, 1.f - (float)p_in_seq / (float)mp.prior_span);
+            const float v = mp.w_entropy * s + mp.w_novelty * (float)novel + mp.w_prior * prior;
+            s = fminf(fmaxf(v, 0.f), 1.f);
+          }
         }
         score[row] = s;
       }
@@ -148,8 +192,28 @@ extern "C" cwl_status cwl_score_tokens(const float* logits, int64_t ld_logits, i
   if (ld_logits < V) return CWL_ERR_SHAPE;
   if ((reinterpret_cast<uintptr_t>(logits) & 3u) != 0) return CWL_ERR_SHAPE;
   int grid = T < (1 << 20) ? T : (1 << 20);
-  cwl::score_rows_kernel<<<grid, cwl::kScoreThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-      logits, ld_logits, T, V, score);
+  cwl::score_rows_kernel<false><<<grid, cwl::kScoreThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      logits, ld_logits, T, V, score, cwl::MixParams{});
+  CWL_CUDA_TRY(cudaGetLastError());
+  return CWL_OK;
+}
+
+extern "C" cwl_status cwl_score_tokens_mixed(const float* logits, int64_t ld_logits, int32_t T, int32_t V,
+                                             const int32_t* token_ids, const int32_t* cu_seqlens, int32_t n_seq,
+                                             const cwl_signal_mix* mix, float* score, void* stream) {
+  if (T < 0 || V < 2 || n_seq < 0 || mix == nullptr) return CWL_ERR_INVALID_ARG;
+  if (mix->ngram < 1 || mix->ngram > 8 || mix->context < 1 || mix->prior_span < 1) return CWL_ERR_INVALID_ARG;
+  if (!(mix->w_entropy >= 0.f) || !(mix->w_novelty >= 0.f) || !(mix->w_prior >= 0.f)) return CWL_ERR_INVALID_ARG;
+  if (T == 0) return CWL_OK;
+  if (logits == nullptr || score == nullptr || token_ids == nullptr || cu_seqlens == nullptr || n_seq < 1)
+    return CWL_ERR_INVALID_ARG;
+  if (ld_logits < V) return CWL_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(logits) & 3u) != 0) return CWL_ERR_SHAPE;
+  cwl::MixParams mp{token_ids, cu_seqlens, n_seq, mix->w_entropy, mix->w_novelty, mix->w_prior,
+                    mix->ngram, mix->context, mix->prior_span};
+  int grid = T < (1 << 20) ? T : (1 << 20);
+  cwl::score_rows_kernel<true><<<grid, cwl::kScoreThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      logits, ld_logits, T, V, score, mp);
   CWL_CUDA_TRY(cudaGetLastError());
   return CWL_OK;
 }
