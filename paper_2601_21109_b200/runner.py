@@ -36,7 +36,7 @@ class HotPath:
     """Device-resident state of one layer's adapted projections plus the scheduler in front."""
 
     def __init__(self, w: Workload, device: str = "cuda", keep_host: bool = False, n_layers: int = 1,
-                 grouped: bool = True, streaming: bool = False):
+                 grouped: bool = True, streaming: bool = False, share_weights: Optional["HotPath"] = None):
         self.grouped = grouped
         # decode with the token-by-token scheduler: every step the cached per-sequence state advances by one
         # token (the rows' scores) and the projections take the row gates it emits instead of a chunk table
@@ -50,15 +50,23 @@ class HotPath:
         self.score = (torch.from_numpy(w.score).to(device) if w.score is not None
                       else torch.empty(w.T, dtype=torch.float32, device=device))
         self.projs: List[DeviceProjection] = []
-        for p in w.projections:
-            self.projs.append(DeviceProjection(
-                p.name, p.d_in, p.d_out, cwl.bf16_from_bits(p.W, device), cwl.bf16_from_bits(p.A, device),
-                cwl.bf16_from_bits(p.B, device), torch.empty(w.T, p.d_out, dtype=torch.bfloat16, device=device)))
+        for i, p in enumerate(w.projections):
+            if share_weights is not None:      # a second slot of activations and outputs over the same weights
+                q = share_weights.projs[i]
+                W, A, B = q.W, q.A, q.B
+            else:
+                W, A, B = cwl.bf16_from_bits(p.W, device), cwl.bf16_from_bits(p.A, device), cwl.bf16_from_bits(p.B, device)
+            self.projs.append(DeviceProjection(p.name, p.d_in, p.d_out, W, A, B,
+                                               torch.empty(w.T, p.d_out, dtype=torch.bfloat16, device=device)))
         # a stack of layers: every layer has its own weights and adapter factors in HBM (distinct memory, so a
         # layer never finds its weights in L2); layers beyond the first hold the first layer's values rolled by
         # one row per layer, which is all a timing run needs
         self.layers: List[List[DeviceProjection]] = [self.projs]
         for l in range(1, n_layers):
+            if share_weights is not None:
+                self.layers.append([DeviceProjection(q.name, q.d_in, q.d_out, q.W, q.A, q.B, p.Y)
+                                    for q, p in zip(share_weights.layers[l], self.projs)])
+                continue
             self.layers.append([DeviceProjection(p.name, p.d_in, p.d_out, torch.roll(p.W, l, 0), torch.roll(p.A, l, 0),
                                                  torch.roll(p.B, l, 1), p.Y) for p in self.projs])
         cap = w.T // max(w.policy.min_len, 1) + self.n_seq + 1
@@ -150,3 +158,58 @@ class HotPath:
         if not self.fixed_table:
             n += self.LAUNCHES_PARTITION
         return n * len(self.layers) + (1 if self.streaming else 0)
+
+
+class HostPipeline:
+    """End-to-end driver for callers whose inputs and results live in host memory.
+
+    Every step copies that step's inputs (activations, logits) from pinned host buffers to the device, runs
+    the hot path and copies all projection outputs back.  Two device slots and three streams (in, compute,
+    out) let step i+1's upload and step i-1's download run under step i's kernels, so a step costs the
+    slowest of the three instead of their sum.  Weights are shared by the slots."""
+
+    def __init__(self, w: Workload, n_layers: int = 1, grouped: bool = True, device: str = "cuda",
+                 first: Optional[HotPath] = None):
+        a = first if first is not None else HotPath(w, device, n_layers=n_layers, grouped=grouped)
+        b = HotPath(w, device, n_layers=n_layers, grouped=grouped, share_weights=a)
+        b.set_thresholds(a.policy.thresholds) if not a.fixed_table and a.logits is not None else None
+        self.slots = [a, b]
+        self.host_X = {d: x.cpu().pin_memory() for d, x in a.X.items()}
+        self.host_logits = a.logits.cpu().pin_memory() if a.logits is not None else None
+        self.host_Y = [[torch.empty(p.Y.shape, dtype=p.Y.dtype).pin_memory() for p in s.projs] for s in self.slots]
+        self.s_in, self.s_run, self.s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+        self.h2d_bytes = sum(x.numel() * x.element_size() for x in self.host_X.values()) + \
+            (self.host_logits.numel() * 4 if self.host_logits is not None else 0)
+        self.d2h_bytes = sum(y.numel() * y.element_size() for y in self.host_Y[0])
+
+    def run(self, steps: int):
+        """Runs `steps` steps; returns (start, end) CUDA events bracketing the first upload and the last download."""
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        uploaded = [None, None]; computed = [None, None]; downloaded = [None, None]
+        self.s_in.wait_stream(torch.cuda.current_stream())
+        start.record(self.s_in)
+        for i in range(steps):
+            k = i & 1
+            slot = self.slots[k]
+            with torch.cuda.stream(self.s_in):
+                if computed[k] is not None:
+                    self.s_in.wait_event(computed[k])           # the slot's inputs were consumed
+                for d, x in self.host_X.items():
+                    slot.X[d].copy_(x, non_blocking=True)
+                if self.host_logits is not None:
+                    slot.logits.copy_(self.host_logits, non_blocking=True)
+                uploaded[k] = torch.cuda.Event(); uploaded[k].record(self.s_in)
+            with torch.cuda.stream(self.s_run):
+                self.s_run.wait_event(uploaded[k])
+                if downloaded[k] is not None:
+                    self.s_run.wait_event(downloaded[k])        # the slot's outputs were read back
+                slot.step()
+                computed[k] = torch.cuda.Event(); computed[k].record(self.s_run)
+            with torch.cuda.stream(self.s_out):
+                self.s_out.wait_event(computed[k])
+                for p, y in zip(slot.projs, self.host_Y[k]):
+                    y.copy_(p.Y, non_blocking=True)
+                downloaded[k] = torch.cuda.Event(); downloaded[k].record(self.s_out)
+        self.s_out.wait_stream(self.s_in); self.s_out.wait_stream(self.s_run)
+        end.record(self.s_out)
+        return start, end
