@@ -276,3 +276,20 @@ def score_tokens_mixed(logits: np.ndarray, token_ids: np.ndarray, cu_seqlens: np
     if rc != 0:
         raise ValueError(f"cwlo_score_tokens_mixed: status {rc}")
     return out
+
+
+# ------------------------------------------------------------------ offline ladder construction (Sec. III-C)
+def _bf16_to_f64(bits: np.ndarray) -> np.ndarray:
+    return (np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def svd_ladder(A: np.ndarray, B: np.ndarray):
+    """SVD-ordered adapter factors (Sec. III-C: the trained update is re-factorised once by SVD so that every
+    prefix of the factors is a usable adapter).  A [d_in, R], B [R, d_out] are bf16 bit patterns.  With
+    A B = U diag(sigma) V^T (singular values in descending order, numpy's LAPACK SVD as the library step) returns
+    (A' = U diag(sigma) [d_in, R], B' = V^T [R, d_out], sigma [R]) in fp64, so that A'[:, :r] B'[:r, :] is the best
+    rank-r approximation of A B for every r (Eckart-Young)."""
+    a, b = _bf16_to_f64(A), _bf16_to_f64(B)
+    R = a.shape[1]
+    U, s, Vt = np.linalg.svd(a @ b, full_matrices=False)
+    return U[:, :R] * s[:R], Vt[:R, :], s[:R]
