@@ -205,6 +205,24 @@ cwl_status cwl_apply_rows(const void* X, int64_t ldx, const void* W, int64_t ldw
                           const cwl_row_gate* gates, void* Y, int64_t ldy,
                           void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream);
 
+/* Offline construction of the rank ladder (Sec. III-C: "obtained once by SVD of the adapter matrix"): re-factorises a
+ * trained adapter so that every prefix of the stored factors is the best adapter of its rank,
+ *   A B = U diag(sigma) V^T,  A_out = U diag(sigma) [d_in, R],  B_out = V^T [R, d_out],  sigma descending,
+ * by two one-sided Jacobi passes in fp64 (no d_in x d_out product, no Gram matrix).  Not on the timed path: the call
+ * synchronises `stream` (once per Jacobi sweep).
+ *   A DEV bf16 [d_in, R], B DEV bf16 [R, d_out]                      inputs, row-major
+ *   A_out / B_out DEV bf16 or NULL; A_out_f32 [d_in, R] / B_out_f32 [R, d_out] / sigma [R] DEV fp32 or NULL (dense)
+ *   workspace DEV, cwl_ladder_workspace_bytes(d_in, d_out, R) bytes, 256-byte aligned;  *sweeps HOST or NULL
+ * Singular vectors are unique up to sign (and up to rotation inside equal singular values); sigma and every prefix
+ * product A_out[:, :r] B_out[:r, :] are unique.
+ * Errors: INVALID_ARG, UNSUPPORTED (R odd, < 2, > CWL_MAX_RANK, > d_in or > d_out), SHAPE, WORKSPACE, CUDA. */
+size_t     cwl_ladder_workspace_bytes(int32_t d_in, int32_t d_out, int32_t R);
+cwl_status cwl_ladder_build(const void* A, int64_t lda, const void* B, int64_t ldb,
+                            int32_t d_in, int32_t d_out, int32_t R,
+                            void* A_out, int64_t lda_out, void* B_out, int64_t ldb_out,
+                            float* A_out_f32, float* B_out_f32, float* sigma,
+                            void* workspace, size_t workspace_bytes, int32_t* sweeps, void* stream);
+
 /* The schedule cwl_apply uses for a shape when `pairs` CTA pairs can be resident (a B200 holds 74): how
  * the output is cut into column tiles (Sec. III-F leaves the kernel schedule open; this is the library's own
  * design), whether the K loop of decode-sized problems is split, and who computes the shrink X A.

@@ -22,7 +22,7 @@ STATUS = {0: "CWL_OK", 1: "CWL_ERR_INVALID_ARG", 2: "CWL_ERR_SHAPE", 3: "CWL_ERR
 EXPORTS = ["cwl_status_string", "cwl_version", "cwl_score_tokens", "cwl_score_tokens_mixed", "cwl_partition_workspace_bytes",
            "cwl_partition", "cwl_apply_workspace_bytes", "cwl_apply", "cwl_apply_grouped_workspace_bytes",
            "cwl_apply_grouped", "cwl_apply_plan", "cwl_stream_state_bytes", "cwl_stream_reset", "cwl_stream_step",
-           "cwl_apply_rows",
+           "cwl_apply_rows", "cwl_ladder_workspace_bytes", "cwl_ladder_build",
            "cwl_apply_noalloc_scratch_need", "cwl_apply_noalloc"]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 
@@ -124,6 +124,12 @@ def lib():
         L.cwl_apply_rows.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
                                      C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                      C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        L.cwl_ladder_workspace_bytes.restype = C.c_size_t
+        L.cwl_ladder_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
+        L.cwl_ladder_build.restype = C.c_int
+        L.cwl_ladder_build.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
+                                       C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                       C.c_void_p, C.c_size_t, C.POINTER(C.c_int32), C.c_void_p]
         L.cwl_apply_plan.restype = C.c_int
         L.cwl_apply_plan.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(CApplyPlanInfo)]
         L.cwl_apply_noalloc_scratch_need.restype = C.c_size_t
@@ -377,6 +383,29 @@ def cwl_apply_rows(X: torch.Tensor, W: torch.Tensor, A: torch.Tensor, B: torch.T
                                                   _p(B), B.stride(0), T, d_in, d_out, R, _p(gates), _p(Y), Y.stride(0),
                                                   _p(workspace), workspace.numel(), _p(status_word), _stream_ptr(stream)))
     return Y
+
+
+def cwl_ladder_build(A: torch.Tensor, B: torch.Tensor, want_f32: bool = True,
+                     stream: Optional[torch.cuda.Stream] = None) -> dict:
+    """SVD-ordered adapter factors of a trained (A [d_in, R], B [R, d_out]) pair, bf16 on the device (offline).
+    Returns dict(A=bf16, B=bf16, sigma=fp32[R], sweeps=int) and, with want_f32, A32 / B32."""
+    assert A.is_cuda and B.is_cuda and A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16
+    assert A.stride(1) == 1 and B.stride(1) == 1
+    d_in, R = A.shape
+    d_out = B.shape[1]
+    out = dict(A=torch.empty(d_in, R, dtype=torch.bfloat16, device=A.device),
+               B=torch.empty(R, d_out, dtype=torch.bfloat16, device=A.device),
+               sigma=torch.empty(R, dtype=torch.float32, device=A.device))
+    if want_f32:
+        out["A32"] = torch.empty(d_in, R, dtype=torch.float32, device=A.device)
+        out["B32"] = torch.empty(R, d_out, dtype=torch.float32, device=A.device)
+    ws = torch.empty(max(int(lib().cwl_ladder_workspace_bytes(d_in, d_out, R)), 256), dtype=torch.uint8, device=A.device)
+    sweeps = C.c_int32(0)
+    _check("cwl_ladder_build", lib().cwl_ladder_build(
+        _p(A), A.stride(0), _p(B), B.stride(0), d_in, d_out, R, _p(out["A"]), R, _p(out["B"]), d_out,
+        _p(out.get("A32")), _p(out.get("B32")), _p(out["sigma"]), _p(ws), ws.numel(), C.byref(sweeps), _stream_ptr(stream)))
+    out["sweeps"] = int(sweeps.value)
+    return out
 
 
 def cwl_apply_noalloc(X: torch.Tensor, W: torch.Tensor, A: Optional[torch.Tensor], B: Optional[torch.Tensor],

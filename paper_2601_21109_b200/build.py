@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcwl.so")
-SOURCES = ["api.cu", "score.cu", "partition.cu", "stream.cu", "apply.cu"]
+SOURCES = ["api.cu", "score.cu", "partition.cu", "stream.cu", "ladder.cu", "apply.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v", "--expt-relaxed-constexpr"]
 
