@@ -4,9 +4,12 @@
 One step = one pass of the whole hot path over one batch of the LLaMA-7B-shaped prefill
 configuration (T = 2048 tokens): token scoring from fp32 logits [T, 32000], adaptive partition and
 rank selection, then the adapted projection for all seven projections (q, k, v, o, gate, up, down)
-with R = 64.  Prints ONE JSON line (see README for the fields).
+with R = 64.  Prints ONE JSON line: metric, value (whole-job tokens/s), ms_per_step, config, clocks, e2e (host
+buffers in and out every step), gpu_launches, roofline (dominant kernel against the measured peaks) and
+cpu_baseline (the fp64 oracle timed on the host cores).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg2|cfg4|cfg1]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload cfg2|cfg3|cfg4|cfg4_stream|cfg5|cfg1] [--layers L] [--no-group] [--lean]
 
 N > 1 runs N independent replicas (one process per GPU, launched with torch.distributed.run); the
 path has no exchange step, so there is no data-path collective: only the timing barrier and the

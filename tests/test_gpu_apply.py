@@ -117,3 +117,30 @@ def test_argument_errors():
         cwl.cwl_apply(X, W, A, B, cwl.DeviceChunkTable(1), 0, workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
     assert e.value.status == 5
     assert cwl.cwl_apply(X[:0], W, A, B, cwl.DeviceChunkTable(1), 0).shape == (0, 64)
+
+
+def test_many_row_tiles_and_widest_rank():
+    # 1300 row tiles of 256 (far more than one wave) on a narrow projection, R = 256: the item loop, the shrink
+    # hand-out and the per-tile flags at scale; sampled rows against the oracle
+    T, d_in, d_out, R = 332_801, 64, 96, 256
+    rng = np.random.default_rng(77)
+    X = wl.normal_bf16(rng, (T, d_in), 1.0)
+    W = wl.normal_bf16(rng, (d_in, d_out), d_in ** -0.5)
+    A = wl.normal_bf16(rng, (d_in, R), d_in ** -0.5)
+    B = wl.normal_bf16(rng, (R, d_out), R ** -0.5)
+    cuts = list(range(1000, T, 1000))
+    n = len(cuts) + 1
+    tab = simple_table(T, cuts, ([256, 64, 0, 128] * n)[:n], ([0.125, 0.5, 0.0, 0.25] * n)[:n], flags=([1, 0, 0, 0, 0] * n)[:n])
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Y = cwl.cwl_apply(dev_bf16(X), dev_bf16(W), dev_bf16(A), dev_bf16(B), dev_table(tab), 8, status_word=status)
+    torch.cuda.synchronize()
+    status_ok(status)
+    rows = np.unique(np.concatenate([[0, 255, 256, T - 2, T - 1], rng.integers(0, T, 200),
+                                     np.array(cuts[:40]), np.array(cuts[:40]) + 3])).astype(np.int32)
+    ref = oracle.apply(X, W, A, B, host_table(tab), 8, rows=rows)
+    check_output(y_to_f64(Y[torch.from_numpy(rows.astype(np.int64)).cuda()]), ref)
+
+
+def test_single_row_and_tiny_widths():
+    run_case(1, 16, 16, 16, simple_table(1, [], [16], [1.0]), 0, seed=78)
+    run_case(5, 48, 32, 32, simple_table(5, [2], [32, 16], [1.0, 2.0]), 2, seed=79)
