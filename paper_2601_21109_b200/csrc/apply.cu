@@ -596,7 +596,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
       if (item.kind == ITEM_PROJECT && pl.split_k == 1) {
         // ---- whole tile: accumulator -> bf16 -> swizzled staging buffer -> TMA store of 32 x 64 boxes ----
         const uint32_t obuf = out_bufs + (uint32_t)(warp - 2) * kOutBufBytes;
-        const int n64 = (item.wt + 63) >> 6;         // a ragged width only occurs at the edge of Y: the store clips it
+        const int n64 = item.wt >> 6;                // whole 64-column chunks go out as TMA boxes
         const int row0 = m_tile * BM + quad * 32;
 #pragma unroll 1
         for (int c64 = chalf; c64 < n64; c64 += 2) {
@@ -623,6 +623,29 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
           if (lane == 0 && row0 < p.T) {
             tma_store_2d(&tm.y[item.proj], obuf, item.n0 + c64 * 64, row0);
             bulk_commit();
+          }
+        }
+        const int rem = item.wt & 63;                // a last chunk of 16, 32 or 48 columns: plain 16-byte stores
+        if (rem != 0 && (n64 & 1) == chalf) {
+#pragma unroll 1
+          for (int h = 0; h * 32 < rem; ++h) {
+            uint32_t v[32];
+            tmem_ld32(t_row + n64 * 64 + h * 32, v);
+            tmem_ld_wait();
+            if (row < p.T) {
+              __nv_bfloat16* out = p.Y[item.proj] + (int64_t)row * p.ldy[item.proj] + item.n0 + n64 * 64 + h * 32;
+#pragma unroll
+              for (int g = 0; g < 4; ++g) {
+                if (h * 32 + g * 8 < rem) {
+                  uint4 q;
+                  q.x = pack_bf16(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
+                  q.y = pack_bf16(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
+                  q.z = pack_bf16(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5]));
+                  q.w = pack_bf16(__uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7]));
+                  *reinterpret_cast<uint4*>(out + g * 8) = q;
+                }
+              }
+            }
           }
         }
         tc_fence_before();
@@ -804,8 +827,10 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
 }
 
 // ------------------------------------------------------------------------------- host: the plan
-// Cost model, in KB of operands a CTA stages: the main loop is bound by operand delivery, so an item
-// costs (K blocks) x (16 KB of rows + 8 KB per right-operand box) plus a per-tile epilogue term.
+// Cost model, in KB of operands a CTA stages per K block: (16 KB of rows + 8 KB per right-operand box), plus a
+// per-tile epilogue term.  (Measured with the loads or the MMAs taken out of the loop, a 512-wide tile is bound by
+// its MMAs, 0.64 us per K block against 0.54 us for its 48 KB of operands; a model that credits narrower tiles
+// with their shorter MMAs picked 464-wide tiles for 4096 columns on 74 pairs and measured 10 % slower.)
 int tile_boxes(int w) {
   const int wa = w < kMmaN ? w : kMmaN, wb = w - wa;
   return boxes_for(wa / 2) + boxes_for(wb / 2);
@@ -853,17 +878,19 @@ Plan search_plan(int T, int d_in, int n_proj, const int* d_out, int R, int pairs
   pl.kb_per_split = ceil_div(pl.nkb0, pl.shrink_splits);
   pl.split_k = 1; pl.kb_per_ksplit = pl.nkb0;
 
-  // ---- column tiling.  Candidates: every projection in tiles of 512 (last one ragged), or with `drop` fewer
-  // wide tiles each and the remaining columns in tiles of w1; or (decode-sized problems: at most half a wave of
+  // ---- column tiling.  Candidates: every projection in tiles of one width (512, 496, ... 128; last one ragged), or
+  // in tiles of 512 with `drop` fewer of them each and the remaining columns in tiles of w1; or (decode-sized problems: at most half a wave of
   // tiles, one width) every tile's K loop split over several pairs.  The busiest pair's cost decides.
   long long best = -1;
   const int narrow_widths[3] = {256, 384, 128};
-  for (int drop = -1; drop <= max_floor; ++drop) {
+  // drop = -1 - u, u = 0..24: one width 512 - 16 u for every tile (each projection's last tile ragged); widths
+  // below 512 are candidates for the split-K form only (measured: they help decode, not prefill)
+  for (int drop = -25; drop <= max_floor; ++drop) {
     for (int wi = 0; wi < 3; ++wi) {
-      int w0 = kMaxTileW, w1 = narrow_widths[wi];
+      int w0 = drop < 0 ? kMaxTileW - 16 * (-1 - drop) : kMaxTileW, w1 = narrow_widths[wi];
       int pw[CWL_MAX_GROUP], pn[CWL_MAX_GROUP], n_wide = 0, n_narrow = 0;
       for (int j = 0; j < n_proj; ++j) {
-        if (drop < 0) { pw[j] = ceil_div(d_out[j], kMaxTileW); pn[j] = 0; }
+        if (drop < 0) { pw[j] = ceil_div(d_out[j], w0); pn[j] = 0; }
         else {
           pw[j] = d_out[j] / kMaxTileW - drop;
           if (pw[j] < 0) pw[j] = 0;
@@ -894,11 +921,13 @@ Plan search_plan(int T, int d_in, int n_proj, const int* d_out, int R, int pairs
         if (s >= 2) {
           const int per = ceil_div(pl.nkb0, s);
           s = ceil_div(pl.nkb0, per);
-          // partial accumulators go out and come back once: about half their size in operand-staging terms
-          const long long c = tile_cost(w0, per + pl.nkb1) + w0 / 2;
+          // every contributor stores and later reads (s-1)/s of a 128 x w0 fp32 accumulator through L2; measured
+          // (~11 us for w0 = 512, s = 3 against 0.8 us per 48 KB K block) that is worth 2 w0 (s-1)/s staged KB
+          const long long c = tile_cost(w0, per + pl.nkb1) + (long long)2 * w0 * (s - 1) / s;
           if (s >= 2 && c < worst) { worst = c; split_k = s; kb_per_ksplit = per; }
         }
       }
+      if (drop < -1 && split_k == 1) break;
       if (best < 0 || worst < best) {
         best = worst;
         pl.w0 = w0; pl.n_wide = n_wide; pl.w1 = w1; pl.n_narrow = n_narrow;
