@@ -223,6 +223,13 @@ cwl_status cwl_ladder_build(const void* A, int64_t lda, const void* B, int64_t l
                             float* A_out_f32, float* B_out_f32, float* sigma,
                             void* workspace, size_t workspace_bytes, int32_t* sweeps, void* stream);
 
+/* Test hook for the failure path of cwl_apply and its variants.  Every device-side wait (mbarrier, H' flag, split-K
+ * counter) is bounded; when one runs out the CTA raises CWL_ERR_TIMEOUT in *status_word (bit 1 << CWL_ERR_TIMEOUT),
+ * drains its copies, frees its tensor memory and returns, so the context stays usable.  This call sets the limit
+ * (ns; <= 0 restores the default of 2 s) and, with withhold_publish != 0, makes the shrink never publish H', so that
+ * the waits on it run out.  Process-wide, not thread-safe, not for production use. */
+void cwl_debug_set(int64_t wait_limit_ns, int32_t withhold_publish);
+
 /* The schedule cwl_apply uses for a shape when `pairs` CTA pairs can be resident (a B200 holds 74): how
  * the output is cut into column tiles (Sec. III-F leaves the kernel schedule open; this is the library's own
  * design), whether the K loop of decode-sized problems is split, and who computes the shrink X A.

@@ -22,7 +22,7 @@ STATUS = {0: "CWL_OK", 1: "CWL_ERR_INVALID_ARG", 2: "CWL_ERR_SHAPE", 3: "CWL_ERR
 EXPORTS = ["cwl_status_string", "cwl_version", "cwl_score_tokens", "cwl_score_tokens_mixed", "cwl_partition_workspace_bytes",
            "cwl_partition", "cwl_apply_workspace_bytes", "cwl_apply", "cwl_apply_grouped_workspace_bytes",
            "cwl_apply_grouped", "cwl_apply_plan", "cwl_stream_state_bytes", "cwl_stream_reset", "cwl_stream_step",
-           "cwl_apply_rows", "cwl_ladder_workspace_bytes", "cwl_ladder_build",
+           "cwl_apply_rows", "cwl_ladder_workspace_bytes", "cwl_ladder_build", "cwl_debug_set",
            "cwl_apply_noalloc_scratch_need", "cwl_apply_noalloc"]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 
@@ -130,6 +130,8 @@ def lib():
         L.cwl_ladder_build.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
                                        C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_size_t, C.POINTER(C.c_int32), C.c_void_p]
+        L.cwl_debug_set.restype = None
+        L.cwl_debug_set.argtypes = [C.c_int64, C.c_int32]
         L.cwl_apply_plan.restype = C.c_int
         L.cwl_apply_plan.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(CApplyPlanInfo)]
         L.cwl_apply_noalloc_scratch_need.restype = C.c_size_t
@@ -406,6 +408,11 @@ def cwl_ladder_build(A: torch.Tensor, B: torch.Tensor, want_f32: bool = True,
         _p(out.get("A32")), _p(out.get("B32")), _p(out["sigma"]), _p(ws), ws.numel(), C.byref(sweeps), _stream_ptr(stream)))
     out["sweeps"] = int(sweeps.value)
     return out
+
+
+def cwl_debug_set(wait_limit_ns: int = 0, withhold_publish: bool = False) -> None:
+    """Test hook: device-side wait limit (<= 0: default) and whether the shrink withholds H' (timeout path)."""
+    lib().cwl_debug_set(int(wait_limit_ns), 1 if withhold_publish else 0)
 
 
 def cwl_apply_noalloc(X: torch.Tensor, W: torch.Tensor, A: Optional[torch.Tensor], B: Optional[torch.Tensor],

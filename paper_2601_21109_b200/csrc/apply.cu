@@ -101,6 +101,8 @@ struct ApplyParams {
   int* sk_counters;        // [2 tiles] split-K partials stored per (tile, CTA rank)
   cwl_chunk_table table;
   const cwl_row_gate* row_gates;   // when set: one descriptor per row instead of the chunk table
+  unsigned long long wait_limit_ns; // limit of every device-side wait
+  int withhold_publish;            // test hook: never publish H', so that the waits on it run out
   int32_t* status_word;
   Plan plan;
 };
@@ -134,6 +136,10 @@ __device__ __forceinline__ unsigned long long global_timer() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
+// The CTA's wait limit in ns sits 12 bytes after its abort flag in shared memory (set once at kernel start).
+__device__ __forceinline__ unsigned long long wait_limit(volatile int* abort_flag) {
+  return *reinterpret_cast<volatile unsigned long long*>(abort_flag + 3);
+}
 // Bounded wait.  Returns false when the limit ran out or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -142,7 +148,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     if ((spins & 255u) == 0) {
       if (*abort_flag) return false;
-      if (global_timer() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+      if (global_timer() - t0 > wait_limit(abort_flag)) { *abort_flag = 1; return false; }
     }
   }
 }
@@ -381,7 +387,7 @@ __device__ __forceinline__ bool wait_word(const int* word, int target, volatile 
     __nanosleep(64);
     if ((spins & 63u) == 0) {
       if (*abort_flag) return false;
-      if (global_timer() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+      if (global_timer() - t0 > wait_limit(abort_flag)) { *abort_flag = 1; return false; }
     }
   }
 }
@@ -432,6 +438,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
     mbar_init(acc_full_bar, 1);
     mbar_init(acc_empty_bar, 2 * kEpiWarps);
     *abort_flag = 0;
+    *reinterpret_cast<volatile unsigned long long*>(abort_flag + 3) = p.wait_limit_ns;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tmap(&tm.x);
     for (int j = 0; j < p.plan.n_proj; ++j) {
@@ -513,7 +520,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
         for (uint32_t back = 1; back <= (uint32_t)n_stages && back <= it_cnt; ++back) {
           const uint32_t j = it_cnt - back;
           unsigned long long t0 = global_timer();
-          while (!mbar_try_wait(full_bar(j % n_stages), (j / n_stages) & 1u) && global_timer() - t0 < kWaitLimitNs) {}
+          while (!mbar_try_wait(full_bar(j % n_stages), (j / n_stages) & 1u) && global_timer() - t0 < wait_limit(abort_flag)) {}
         }
       }
     }
@@ -781,7 +788,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
       __threadfence();                               // this thread's H' / partial stores, device-wide
       epilogue_barrier();
       if (direct) {
-        if (epi_tid == 0) st_release(p.flags + m_tile, 1);
+        if (epi_tid == 0 && !p.withhold_publish) st_release(p.flags + m_tile, 1);
         continue;
       }
       if (epi_tid == 0) *epi_last = (atomicAdd(p.counters + m_tile, 1) == pl.shrink_splits - 1);
@@ -810,7 +817,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
       }
       __threadfence();
       epilogue_barrier();
-      if (epi_tid == 0) st_release(p.flags + m_tile, 1);
+      if (epi_tid == 0 && !p.withhold_publish) st_release(p.flags + m_tile, 1);
     }
     if (lane == 0) bulk_wait_all();                  // this warp's TMA stores have left shared memory and landed
   }
@@ -1123,6 +1130,10 @@ int max_pairs() {
   return n;
 }
 
+// process-wide test hook state (cwl_debug_set)
+unsigned long long g_wait_limit_ns = kWaitLimitNs;
+int g_withhold_publish = 0;
+
 struct ApplyWorkspace { __nv_bfloat16* Hg; float* partial; float* sk_partial; int* sync; size_t sync_bytes; };
 
 // Carves the workspace for a plan.
@@ -1223,6 +1234,7 @@ cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* pr
   p.Hg = ws.Hg; p.partial = ws.partial; p.sk_partial = ws.sk_partial;
   p.counters = ws.sync; p.flags = ws.sync + 2 * pl.n_m_pairs; p.sk_counters = ws.sync + 4 * pl.n_m_pairs;
   p.table = table; p.row_gates = row_gates; p.status_word = status_word;
+  p.wait_limit_ns = g_wait_limit_ns; p.withhold_publish = g_withhold_publish;
   p.plan = pl;
 
   // the counters and flags are the only words that must start at zero
@@ -1261,6 +1273,11 @@ extern "C" size_t cwl_apply_workspace_bytes(int32_t T, int32_t d_in, int32_t d_o
   cwl::ApplyWorkspace w;
   const cwl::Plan pl = cwl::make_plan(T, d_in, 1, &d_out, R, cwl::max_pairs(), true);
   return cwl::carve_apply(w, nullptr, pl, T, R);
+}
+
+extern "C" void cwl_debug_set(int64_t wait_limit_ns, int32_t withhold_publish) {
+  cwl::g_wait_limit_ns = wait_limit_ns > 0 ? (unsigned long long)wait_limit_ns : cwl::kWaitLimitNs;
+  cwl::g_withhold_publish = withhold_publish != 0 ? 1 : 0;
 }
 
 extern "C" cwl_status cwl_apply_plan(int32_t T, int32_t d_in, int32_t d_out, int32_t R, int32_t pairs,
