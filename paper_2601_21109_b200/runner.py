@@ -151,6 +151,17 @@ class HotPath:
                 self.partition_step()
             self.apply_step(layer=layer)
 
+    def capture(self) -> "torch.cuda.CUDAGraph":
+        """Records one step (every launch and the few-hundred-byte memsets of the sync words) into a CUDA graph.
+        The library allocates nothing and synchronises nothing on this path; run one ordinary step first so that
+        tensor-map descriptors, plans and kernel attributes are set up outside the capture."""
+        self.step()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.step()
+        return graph
+
     def launches_per_step(self) -> int:
         n = self.LAUNCHES_APPLY * len(self.launch_groups())
         if self.logits is not None:
