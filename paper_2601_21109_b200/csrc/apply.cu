@@ -60,7 +60,7 @@ constexpr int kABytes = BM * BK * 2;          // 16 KB: this CTA's 128 rows of t
 constexpr int kBoxBytes = kBoxCols * BK * 2;  // 8 KB
 constexpr int kMaxStages = 8;
 constexpr int kRingBytes = 192 * 1024;
-constexpr int kOutBufBytes = 4096;  // per epilogue warp: 32 rows x 64 bf16 columns staged for a TMA store
+constexpr int kOutBufBytes = 4096;  // per epilogue warp: 32 rows x 64 bf16 columns staged for row-contiguous stores
 constexpr int kThreads = 320;       // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: epilogue
 constexpr int kEpiThreads = 256;
 constexpr int kEpiWarps = 8;
@@ -112,7 +112,7 @@ struct ApplyParams {
 // Tensor maps of one launch: X and H' are shared, the rest is per projection.
 struct GroupMaps {
   CUtensorMap x, h;
-  CUtensorMap w[CWL_MAX_GROUP], a[CWL_MAX_GROUP], b[CWL_MAX_GROUP], y[CWL_MAX_GROUP];
+  CUtensorMap w[CWL_MAX_GROUP], a[CWL_MAX_GROUP], b[CWL_MAX_GROUP];
 };
 
 // ------------------------------------------------------------------------------------------ PTX
@@ -161,16 +161,13 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(map), "r"(leader_bar), "r"(x), "r"(y) : "memory");
 }
-// TMA store of a staged box (shared -> global); rows and columns outside the tensor are clipped
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-               ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -412,7 +409,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;     // swizzled tiles need 1024-byte alignment
   uint8_t* base_ptr = smem_raw + (base - raw);
-  const uint32_t out_bufs = base + kRingBytes;      // 1024-byte aligned: the TMA store reads it with the 128-byte swizzle
+  const uint32_t out_bufs = base + kRingBytes;      // per-warp staging buffers of the epilogue
   const uint32_t bars = out_bufs + L::kOutBytes;
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
@@ -445,7 +442,6 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
     prefetch_tmap(&tm.x);
     for (int j = 0; j < p.plan.n_proj; ++j) {
       prefetch_tmap(&tm.w[j]);
-      prefetch_tmap(&tm.y[j]);
       if (p.R > 0) { prefetch_tmap(&tm.a[j]); prefetch_tmap(&tm.b[j]); }
     }
     if (p.R > 0) prefetch_tmap(&tm.h);
@@ -603,14 +599,14 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
       const int n_chunks = (item.wt + 31) >> 5;
 
       if (item.kind == ITEM_PROJECT && pl.split_k == 1) {
-        // ---- whole tile: accumulator -> bf16 -> swizzled staging buffer -> TMA store of 32 x 64 boxes ----
+        // ---- whole tile: accumulator -> bf16 -> swizzled staging buffer (a lane holds a row) -> read back so that
+        // a warp instruction stores four whole 128-byte row segments ----
         const uint32_t obuf = out_bufs + (uint32_t)(warp - 2) * kOutBufBytes;
-        const int n64 = item.wt >> 6;                // whole 64-column chunks go out as TMA boxes
+        const int n64 = item.wt >> 6;                // whole 64-column chunks
         const int row0 = m_tile * BM + quad * 32;
 #pragma unroll 1
         for (int c64 = chalf; c64 < n64; c64 += 2) {
-          if (lane == 0) bulk_wait_read();           // the previous store has finished reading this buffer
-          __syncwarp();
+          __syncwarp();                              // every lane has read the previous chunk back
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
             uint32_t v[32];
@@ -627,11 +623,14 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
               st_shared_v4(obuf + lane * 128 + ((piece ^ (lane & 7)) << 4), q);
             }
           }
-          fence_proxy_async();                       // the staged rows, visible to the TMA engine
           __syncwarp();
-          if (lane == 0 && row0 < p.T) {
-            tma_store_2d(&tm.y[item.proj], obuf, item.n0 + c64 * 64, row0);
-            bulk_commit();
+          __nv_bfloat16* out = p.Y[item.proj] + item.n0 + c64 * 64 + (lane & 7) * 8;
+          const int64_t ldy = p.ldy[item.proj];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const int r = (lane >> 3) + 4 * k;       // lanes 8j..8j+7 take the eight pieces of row r
+            const uint4 q = ld_shared_v4(obuf + r * 128 + (((lane & 7) ^ (r & 7)) << 4));
+            if (row0 + r < p.T) *reinterpret_cast<uint4*>(out + (int64_t)(row0 + r) * ldy) = q;
           }
         }
         const int rem = item.wt & 63;                // a last chunk of 16, 32 or 48 columns: plain 16-byte stores
@@ -821,7 +820,6 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
       epilogue_barrier();
       if (epi_tid == 0 && !p.withhold_publish) st_release(p.flags + m_tile, 1);
     }
-    if (lane == 0) bulk_wait_all();                  // this warp's TMA stores have left shared memory and landed
   }
 
   // ---------------------------------------------------------------------- teardown
@@ -1220,7 +1218,6 @@ cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* pr
   if (adapter && !make_map(&maps.h, ws.Hg, (uint64_t)n_proj * R, (uint64_t)T, (uint64_t)n_proj * R, BK, BM)) return CWL_ERR_CUDA;
   for (int j = 0; j < n_proj; ++j) {
     const cwl_projection& q = proj[j];
-    if (!make_map(&maps.y[j], q.Y, (uint64_t)q.d_out, (uint64_t)T, (uint64_t)q.ldy, 64, 32)) return CWL_ERR_CUDA;
     if (!make_map(&maps.w[j], q.W, (uint64_t)q.d_out, (uint64_t)d_in, (uint64_t)q.ldw, kBoxCols, BK)) return CWL_ERR_CUDA;
     maps.a[j] = maps.w[j]; maps.b[j] = maps.w[j];   // never dereferenced when R == 0
     if (adapter) {
