@@ -145,14 +145,14 @@ cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64_t ldw,
 /* Several adapted projections of the SAME rows in one launch (Sec. III-F: the adapter sits on every attention and
  * MLP projection; q, k, v read one activation, gate and up another).  Projection j computes
  *   Y_j = X W_j + gated (X A_j) B_j
- * exactly as cwl_apply does, with the chunk table, window, d_in and R shared by the group.  One pass over X serves
- * all shrinks, and the output tiles of all projections are scheduled together, which fills the last wave of tiles
- * better than separate calls.  Meant for prefill-sized T; decode-sized T is better served by separate cwl_apply
+ * exactly as cwl_apply does, with the chunk table, window, d_in and R shared by the group.  The output tiles and the
+ * shrink work of all projections are scheduled together, which fills the last wave of tiles better than separate
+ * calls.  Meant for prefill-sized T; decode-sized T is better served by separate cwl_apply
  * calls, whose K loop is split.
  *   proj        HOST array of n_proj descriptors (1 <= n_proj <= CWL_MAX_GROUP), copied at call time; all pointers
  *               inside are DEV.  Either every projection has A and B, or none has.
  *   workspace   DEV, at least cwl_apply_grouped_workspace_bytes(T, d_in, n_proj, d_out[], R) bytes, 256-byte aligned
- * Shape rules and errors as for cwl_apply, plus UNSUPPORTED when n_proj * R > 512. */
+ * Shape rules and errors as for cwl_apply. */
 #define CWL_MAX_GROUP 4
 typedef struct {
   const void* W; int64_t ldw;   /* DEV bf16 [d_in, d_out] */

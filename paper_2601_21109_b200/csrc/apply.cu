@@ -13,8 +13,8 @@
 // 0.54 us of operand delivery per K block); the real kernel runs within 3-10 % of its MMAs alone.
 //
 // Work items of a pair, in order:
-//   SHRINK   P[split] = X[:, split of d_in] A[split, :]  at the full ladder rank R (fp32 partials when
-//            d_in is split); the CTA that completes a row tile's last split sums the partials, applies
+//   SHRINK   P[split] = X[:, split of d_in] A[split, :]  at the full ladder rank R, one item per projection
+//            (fp32 partials when d_in is split); the CTA that completes a row tile's last split sums the partials, applies
 //            the per-row gate (rank mask, scale and cross-fade weight from the chunk table, expanded per
 //            row in shared memory) and publishes H' = bf16(g * X A) with a release flag.  The host-side
 //            plan hands shrink items to the pairs with the lightest projection load.
@@ -22,7 +22,7 @@
 //            accumulator (the TMA producer acquires the row tile's flag before its first H' load).
 //            Column tiles come in two widths (wide ones first, then narrower ones that fill the last
 //            wave); items are dealt round-robin.  Up to four projections that read the same rows can share
-//            one launch (their tiles are dealt together, their shrinks share the pass over X).  When the whole problem is a fraction of one wave
+//            one launch (their tiles and shrink items are dealt together).  When the whole problem is a fraction of one wave
 //            (decode-sized T) the K loop of each tile is split over several pairs instead: each writes
 //            an fp32 partial, and once all of a tile's partials are in, every contributor reduces its
 //            share of the tile's columns and writes Y.
@@ -98,8 +98,8 @@ struct ApplyParams {
   __nv_bfloat16* Hg;       // [T, RT] gated shrink outputs
   float* partial;          // [shrink_splits, 128-row tiles, RT / 4, 128, 4] fp32 partial shrink sums
   float* sk_partial;       // [tiles * split_k * 2, 128, w0] fp32 partial accumulators of split-K items
-  int* counters;           // [2 n_m_pairs] shrink splits finished per 128-row tile
-  int* flags;              // [2 n_m_pairs] 1 once H' of the 128-row tile is published
+  int* counters;           // [2 n_m_pairs][n_proj] shrink splits finished per (128-row tile, projection)
+  int* flags;              // [2 n_m_pairs][n_proj] 1 once that projection's H' columns of the row tile are published
   int* sk_counters;        // [2 tiles] split-K partials stored per (tile, CTA rank)
   cwl_chunk_table table;
   const cwl_row_gate* row_gates;   // when set: one descriptor per row instead of the chunk table
@@ -305,9 +305,11 @@ __device__ __forceinline__ bool get_item(int i, int b, int sh_begin, const Apply
   const Plan& pl = p.plan;
   const int my_shrink = pl.sh_count[b];
   if (i < my_shrink) {
-    const int s = sh_begin + i;
-    it.kind = ITEM_SHRINK; it.m_pair = s / pl.shrink_splits; it.split = s - it.m_pair * pl.shrink_splits;
-    it.n0 = 0; it.wt = p.RT; it.tile = 0; it.proj = 0;
+    const int s = sh_begin + i, per_row = pl.n_proj * pl.shrink_splits;   // one item per (row tile, projection, split)
+    it.kind = ITEM_SHRINK; it.m_pair = s / per_row;
+    const int rem = s - it.m_pair * per_row;
+    it.proj = rem / pl.shrink_splits; it.split = rem - it.proj * pl.shrink_splits;
+    it.n0 = 0; it.wt = p.R; it.tile = 0;
     it.kb0 = it.split * pl.kb_per_split;
     it.n_blk0 = min(pl.nkb0, it.kb0 + pl.kb_per_split) - it.kb0;
     it.n_blk1 = 0;
@@ -472,31 +474,28 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
       for (int i = 0; ok && get_item(i, pair, sh_begin, p, item); ++i) {
         const bool shrink = item.kind == ITEM_SHRINK;
         const int m_tile = item.m_pair * 2 + (int)rank;       // this CTA's 128-row tile
-        // columns of the right operand this CTA supplies: its half of each MMA's columns.  A shrink item runs
-        // one MMA of N = R per projection (their A factors are separate matrices); a projection tile runs one or two.
-        const int ca = shrink ? (p.R >> 1) : (item.wa >> 1), cb = shrink ? 0 : (item.wb >> 1);
+        // columns of the right operand this CTA supplies: its half of each MMA's columns (a shrink item runs one
+        // MMA of N = R against its projection's A, a projection tile one or two MMAs)
+        const int ca = item.wa >> 1, cb = item.wb >> 1;
         const int boxes_a = boxes_for(ca), boxes_b = boxes_for(cb);
-        const int col_a = shrink ? (int)rank * ca : item.n0 + (int)rank * ca;
+        const int col_a = item.n0 + (int)rank * ca;
         const int col_b = item.n0 + item.wa + (int)rank * cb;
-        const int n_boxes = shrink ? pl.n_proj * boxes_a : boxes_a + boxes_b;
+        const int n_boxes = boxes_a + boxes_b;
         const uint32_t tx_pair = 2u * (kABytes + n_boxes * kBoxBytes);
         // this lane's box (lanes 1..n_boxes): source matrix in the d_in blocks and in the R blocks, column, slot
         const int bi = lane - 1;
         const bool has_box = bi >= 0 && bi < n_boxes;
-        const CUtensorMap* map0 = &tm.w[item.proj];
+        const CUtensorMap* map0 = shrink ? &tm.a[item.proj] : &tm.w[item.proj];
         const CUtensorMap* map1 = &tm.b[item.proj];
         int box_x = 0;
-        if (has_box) {
-          if (shrink) { map0 = &tm.a[bi / boxes_a]; box_x = col_a + (bi % boxes_a) * kBoxCols; }
-          else box_x = bi < boxes_a ? col_a + bi * kBoxCols : col_b + (bi - boxes_a) * kBoxCols;
-        }
+        if (has_box) box_x = bi < boxes_a ? col_a + bi * kBoxCols : col_b + (bi - boxes_a) * kBoxCols;
         const int n_blk = item.n_blk0 + item.n_blk1;
         for (int b = 0; b < n_blk; ++b, ++it_cnt) {
           bool step_ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag);
           const bool phase1 = b >= item.n_blk0;
           if (phase1 && b == item.n_blk0) {
             // H' of this CTA's row tile must have been published by whoever finished its shrink
-            if (lane == 0 && step_ok) step_ok = wait_word(p.flags + m_tile, 1, abort_flag);
+            if (lane == 0 && step_ok) step_ok = wait_word(p.flags + m_tile * pl.n_proj + item.proj, 1, abort_flag);
             fence_proxy_async();
           }
           if (!__all_sync(0xffffffffu, step_ok)) { ok = false; break; }
@@ -530,11 +529,9 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
       bool ok = true;
       Item item;
       for (int i = 0; ok && get_item(i, pair, sh_begin, p, item); ++i, ++local) {
-        const bool shrink = item.kind == ITEM_SHRINK;
-        const uint32_t idesc_a = make_idesc(2 * BM, shrink ? p.R : item.wa);
+        const uint32_t idesc_a = make_idesc(2 * BM, item.wa);
         const uint32_t idesc_b = make_idesc(2 * BM, item.wb > 0 ? item.wb : 16);
         const uint32_t sb_off_b = (uint32_t)boxes_for(item.wa >> 1) * kBoxBytes;
-        const uint32_t sb_step_r = (uint32_t)boxes_for(p.R >> 1) * kBoxBytes;   // shrink: boxes of one projection's A
         if (!mbar_wait(acc_empty_bar, (local & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const int n_blk = item.n_blk0 + item.n_blk1;
@@ -551,12 +548,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
             const uint64_t da = make_smem_desc(sa + kk * (UMMA_K * 2), 16, 1024);
             const uint64_t db = make_smem_desc(sb + kk * (UMMA_K * 128), kBoxBytes, 1024);
             umma_bf16_pair(tmem_base, da, db, idesc_a, acc_flag);
-            if (shrink) {
-              for (int q = 1; q < pl.n_proj; ++q) {
-                const uint64_t dq = make_smem_desc(sb + q * sb_step_r + kk * (UMMA_K * 128), kBoxBytes, 1024);
-                umma_bf16_pair(tmem_base + q * p.R, da, dq, idesc_a, acc_flag);
-              }
-            } else if (item.wb > 0) {
+            if (item.wb > 0) {
               const uint64_t db2 = make_smem_desc(sb + sb_off_b + kk * (UMMA_K * 128), kBoxBytes, 1024);
               umma_bf16_pair(tmem_base + kMmaN, da, db2, idesc_b, acc_flag);
             }
@@ -750,6 +742,8 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
       // ---- shrink item ----
       const bool direct = pl.shrink_splits == 1;     // no partials: gate straight from the accumulator
       const RowGate g = gates[row_in_tile];          // written before the barriers above
+      const int sync_idx = m_tile * pl.n_proj + item.proj;   // counter and flag of this (row tile, projection)
+      const int hcol = item.proj * p.R;              // this projection's columns of H'
 #pragma unroll 1
       for (int cc = chalf; cc < n_chunks; cc += 2) {
         const int col = cc * 32;
@@ -758,19 +752,19 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
         tmem_ld_wait();
         if (!direct) {
           // partial layout [split][128-row tile][column group of 4][128 rows][4]: contiguous per warp store
-          float* out = p.partial + (((int64_t)(item.split * 2 * pl.n_m_pairs + m_tile) * (p.RT >> 2) + cc * 8) * BM + row_in_tile) * 4;
+          float* out = p.partial + (((int64_t)(item.split * 2 * pl.n_m_pairs + m_tile) * (p.RT >> 2) + (hcol >> 2) + cc * 8) * BM + row_in_tile) * 4;
 #pragma unroll
           for (int q4 = 0; q4 < 8; ++q4) {
-            if (col + q4 * 4 < p.RT)
+            if (col + q4 * 4 < p.R)
               *reinterpret_cast<uint4*>(out + q4 * BM * 4) = make_uint4(v[q4 * 4 + 0], v[q4 * 4 + 1], v[q4 * 4 + 2], v[q4 * 4 + 3]);
           }
         } else if (row < p.T) {
           {
-            __nv_bfloat16* out = p.Hg + (int64_t)row * p.RT + col;
+            __nv_bfloat16* out = p.Hg + (int64_t)row * p.RT + hcol + col;
 #pragma unroll
             for (int q8 = 0; q8 < 4; ++q8) {
-              if (col + q8 * 8 < p.RT) {
-                const int j = (col + q8 * 8) % p.R;      // rank index inside its projection (R is a multiple of 8)
+              if (col + q8 * 8 < p.R) {
+                const int j = col + q8 * 8;              // rank index (R is a multiple of 8)
                 uint4 q;
                 q.x = pack_bf16(__uint_as_float(v[q8 * 8 + 0]) * gate_at(g, j + 0), __uint_as_float(v[q8 * 8 + 1]) * gate_at(g, j + 1));
                 q.y = pack_bf16(__uint_as_float(v[q8 * 8 + 2]) * gate_at(g, j + 2), __uint_as_float(v[q8 * 8 + 3]) * gate_at(g, j + 3));
@@ -789,23 +783,23 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
       __threadfence();                               // this thread's H' / partial stores, device-wide
       epilogue_barrier();
       if (direct) {
-        if (epi_tid == 0 && !p.withhold_publish) st_release(p.flags + m_tile, 1);
+        if (epi_tid == 0 && !p.withhold_publish) st_release(p.flags + sync_idx, 1);
         continue;
       }
-      if (epi_tid == 0) *epi_last = (atomicAdd(p.counters + m_tile, 1) == pl.shrink_splits - 1);
+      if (epi_tid == 0) *epi_last = (atomicAdd(p.counters + sync_idx, 1) == pl.shrink_splits - 1);
       epilogue_barrier();
       if (*epi_last == 0) continue;
-      // this CTA completed its row tile: sum the partials, gate, publish H'
+      // this CTA completed its projection's share of the row tile: sum the partials, gate, publish H'
       __threadfence();
-      const int quads = p.RT >> 2;                   // float4 groups per row
+      const int quads = p.R >> 2;                    // float4 groups per row of this projection
       const int64_t split_stride = (int64_t)2 * pl.n_m_pairs * p.RT * BM;
       for (int idx = epi_tid; idx < BM * quads; idx += kEpiThreads) {
-        const int r = idx & (BM - 1), cg = idx >> 7, jt = cg << 2, j0 = jt % p.R;   // column, rank index in its projection
+        const int r = idx & (BM - 1), cg = idx >> 7, j0 = cg << 2;   // rank index
         const int t = m_tile * BM + r;
         if (t >= p.T) continue;
         const RowGate gr = gates[r];
         float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-        const float* src = p.partial + (((int64_t)m_tile * quads + cg) * BM + r) * 4;
+        const float* src = p.partial + (((int64_t)m_tile * (p.RT >> 2) + (hcol >> 2) + cg) * BM + r) * 4;
 #pragma unroll 4
         for (int s = 0; s < pl.shrink_splits; ++s) {
           const float4 x = __ldcg(reinterpret_cast<const float4*>(src + s * split_stride));
@@ -814,11 +808,11 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
         uint2 o;
         o.x = pack_bf16(sum.x * gate_at(gr, j0), sum.y * gate_at(gr, j0 + 1));
         o.y = pack_bf16(sum.z * gate_at(gr, j0 + 2), sum.w * gate_at(gr, j0 + 3));
-        *reinterpret_cast<uint2*>(p.Hg + (int64_t)t * p.RT + jt) = o;
+        *reinterpret_cast<uint2*>(p.Hg + (int64_t)t * p.RT + hcol + j0) = o;
       }
       __threadfence();
       epilogue_barrier();
-      if (epi_tid == 0 && !p.withhold_publish) st_release(p.flags + m_tile, 1);
+      if (epi_tid == 0 && !p.withhold_publish) st_release(p.flags + sync_idx, 1);
     }
   }
 
@@ -949,13 +943,13 @@ Plan search_plan(int T, int d_in, int n_proj, const int* d_out, int R, int pairs
   pl.pairs = n_items < pairs ? n_items : pairs;
   if (R > 0 && pl.pairs < pairs) {
     // pairs beyond the projection items exist only to carry shrink items
-    const int n_shrink = pl.n_m_pairs * pl.shrink_splits;
+    const int n_shrink = pl.n_m_pairs * n_proj * pl.shrink_splits;
     pl.pairs = n_items + n_shrink < pairs ? n_items + n_shrink : pairs;
   }
 
   pl.boxes = tile_boxes(pl.w0);
   if (pl.n_narrow > 0 && tile_boxes(pl.w1) > pl.boxes) pl.boxes = tile_boxes(pl.w1);
-  if (R > 0 && n_proj * boxes_for(R / 2) > pl.boxes) pl.boxes = n_proj * boxes_for(R / 2);
+  if (R > 0 && boxes_for(R / 2) > pl.boxes) pl.boxes = boxes_for(R / 2);
   pl.stages = kRingBytes / (kABytes + pl.boxes * kBoxBytes);
   if (pl.stages > kMaxStages) pl.stages = kMaxStages;
 
@@ -975,12 +969,12 @@ Plan search_plan(int T, int d_in, int n_proj, const int* d_out, int R, int pairs
       if (want > pl.nkb0) break;
       const int per = ceil_div(pl.nkb0, want), splits = ceil_div(pl.nkb0, per);
       const size_t RT = (size_t)n_proj * R;
-      const size_t scratch = (size_t)T * RT * 2 + (size_t)splits * pl.n_m_pairs * 2 * BM * RT * 4 + 4096 + 16 * (size_t)pl.n_m_pairs;
+      const size_t scratch = (size_t)T * RT * 2 + (size_t)splits * pl.n_m_pairs * 2 * BM * RT * 4 + 4096 + 16 * (size_t)pl.n_m_pairs * n_proj;
       if (scratch_limit > 0 && splits > 1 && scratch > scratch_limit) continue;
       // measured: a shrink K block costs about 1.3x its staged bytes (narrow MMAs), an item ~4 us of fixed cost
-      const long long cs = (long long)per * (16 + 8 * n_proj * boxes_for(R / 2)) * 13 / 10 + 250;
+      const long long cs = (long long)per * (16 + 8 * boxes_for(R / 2)) * 13 / 10 + 250;
       const long long due = first_tile * 4 / 5;
-      const int n_shrink = pl.n_m_pairs * splits;
+      const int n_shrink = pl.n_m_pairs * n_proj * splits;   // one item per (row-tile pair, projection, split)
       uint16_t count[kPairsPlanned];
       long long shrink_time[kPairsPlanned];
       for (int g = 0; g < pl.pairs; ++g) { load[g] = base_load[g]; count[g] = 0; shrink_time[g] = 0; }
@@ -1150,8 +1144,8 @@ size_t carve_apply(ApplyWorkspace& w, char* base, const Plan& pl, int T, int R) 
   const size_t n_tiles = (size_t)pl.n_m_pairs * pl.n_wide;              // split plans have one tile width
   if (split) off = up(off + n_tiles * pl.split_k * 2 * BM * pl.w0 * sizeof(float));
   w.sync = reinterpret_cast<int*>(base ? base + off : nullptr);
-  // shrink counters [2 n_m], H' flags [2 n_m], split-K counters [2 tiles]
-  w.sync_bytes = sizeof(int) * ((size_t)4 * pl.n_m_pairs + (split ? 2 * n_tiles : 0));
+  // shrink counters [2 n_m][n_proj], H' flags [2 n_m][n_proj], split-K counters [2 tiles]
+  w.sync_bytes = sizeof(int) * ((size_t)4 * pl.n_m_pairs * pl.n_proj + (split ? 2 * n_tiles : 0));
   off = up(off + w.sync_bytes);
   return off < 256 ? 256 : off;
 }
@@ -1170,7 +1164,7 @@ cwl_status check_group(const void* X, int64_t ldx, const cwl_projection* proj, i
   if (with != 0 && with != n_proj) return CWL_ERR_INVALID_ARG;   // adapters on all projections of a group or on none
   adapter = with == n_proj;
   if (d_in % 16 != 0) return CWL_ERR_UNSUPPORTED;
-  if (adapter && (R % 16 != 0 || R > CWL_MAX_RANK || n_proj * R > kMaxTileW)) return CWL_ERR_UNSUPPORTED;
+  if (adapter && (R % 16 != 0 || R > CWL_MAX_RANK)) return CWL_ERR_UNSUPPORTED;
   if (ldx < d_in || ldx % 8 != 0 || !aligned16(X)) return CWL_ERR_SHAPE;
   for (int j = 0; j < n_proj; ++j) {
     const cwl_projection& q = proj[j];
@@ -1231,7 +1225,7 @@ cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* pr
   p.window = window;
   for (int j = 0; j < n_proj; ++j) { p.Y[j] = static_cast<__nv_bfloat16*>(proj[j].Y); p.ldy[j] = proj[j].ldy; }
   p.Hg = ws.Hg; p.partial = ws.partial; p.sk_partial = ws.sk_partial;
-  p.counters = ws.sync; p.flags = ws.sync + 2 * pl.n_m_pairs; p.sk_counters = ws.sync + 4 * pl.n_m_pairs;
+  p.counters = ws.sync; p.flags = ws.sync + 2 * pl.n_m_pairs * n_proj; p.sk_counters = ws.sync + 4 * pl.n_m_pairs * n_proj;
   p.table = table; p.row_gates = row_gates; p.status_word = status_word;
   p.wait_limit_ns = g_wait_limit_ns; p.withhold_publish = g_withhold_publish;
   p.plan = pl;

@@ -50,13 +50,19 @@ def test_two_projections_rank16_and_different_widths():
     run_group(T, 128, [1040, 64], 16, tab, 4, seed=32)
 
 
-def test_four_projections_R128_fills_tensor_memory():
+def test_four_projections_at_rank_128():
     T = 160
     tab = table_for(T, [50, 100], [128, 64, 16], [0.25, 0.5, 2.0])
     run_group(T, 256, [128, 144, 160, 176], 128, tab, 6, seed=33)
 
 
-def test_dense_group():
+def test_three_projections_at_the_largest_rank_and_a_split_shrink():
+    T = 200                                                    # d_in = 2048, small T: the shrink is split along d_in
+    tab = table_for(T, [60, 130], [256, 96, 32], [0.125, 0.5, 1.0])
+    run_group(T, 2048, [128, 64, 192], 256, tab, 8, seed=36)
+
+
+def test_group_without_adapter():
     run_group(300, 208, [336, 528], 16, None, 0, seed=34, adapter=False)
 
 
@@ -75,9 +81,9 @@ def test_group_of_one_equals_cwl_apply():
 def test_argument_errors():
     X = torch.zeros(8, 64, dtype=torch.bfloat16, device="cuda")
     W = torch.zeros(64, 64, dtype=torch.bfloat16, device="cuda")
-    A = torch.zeros(64, 256, dtype=torch.bfloat16, device="cuda")
-    B = torch.zeros(256, 64, dtype=torch.bfloat16, device="cuda")
-    with pytest.raises(cwl.CwlError) as e:                    # 3 x 256 shrink columns do not fit tensor memory
+    A = torch.zeros(64, 40, dtype=torch.bfloat16, device="cuda")
+    B = torch.zeros(40, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(cwl.CwlError) as e:                    # the ladder's top rank must be a multiple of 16
         cwl.cwl_apply_grouped(X, [W] * 3, [A] * 3, [B] * 3, cwl.DeviceChunkTable(1), 0)
     assert e.value.status == 3
     with pytest.raises(cwl.CwlError) as e:                    # more projections than a group holds
