@@ -39,10 +39,13 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <atomic>
+#include <chrono>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <random>
 #include <unordered_map>
 
 #include "cwl_common.cuh"
@@ -98,9 +101,12 @@ struct ApplyParams {
   __nv_bfloat16* Hg;       // [T, RT] gated shrink outputs
   float* partial;          // [shrink_splits, 128-row tiles, RT / 4, 128, 4] fp32 partial shrink sums
   float* sk_partial;       // [tiles * split_k * 2, 128, w0] fp32 partial accumulators of split-K items
-  int* counters;           // [2 n_m_pairs][n_proj] shrink splits finished per (128-row tile, projection)
-  int* flags;              // [2 n_m_pairs][n_proj] 1 once that projection's H' columns of the row tile are published
-  int* sk_counters;        // [2 tiles] split-K partials stored per (tile, CTA rank)
+  // Sync words are 64 bits: (epoch of the launch << 8) | count.  A word that carries another epoch (left by an earlier
+  // launch, or never written) counts as zero, so nothing has to be cleared between launches.
+  unsigned long long* counters;     // [2 n_m_pairs][n_proj] shrink splits finished per (128-row tile, projection)
+  unsigned long long* flags;        // [2 n_m_pairs][n_proj] 1 once that projection's H' columns of the row tile are published
+  unsigned long long* sk_counters;  // [2 tiles] split-K partials stored per (tile, CTA rank)
+  unsigned long long epoch;         // this launch's tag, already shifted: low 8 bits zero
   cwl_chunk_table table;
   const cwl_row_gate* row_gates;   // when set: one descriptor per row instead of the chunk table
   unsigned long long wait_limit_ns; // limit of every device-side wait
@@ -240,13 +246,28 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 __device__ __forceinline__ void epilogue_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-__device__ __forceinline__ int ld_acquire(const int* p) {
-  int v;
-  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+__device__ __forceinline__ unsigned long long ld_acquire(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ void st_release(int* p, int v) {
-  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+__device__ __forceinline__ void st_release(unsigned long long* p, unsigned long long v) {
+  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+// count carried by a sync word for the launch tagged `epoch` (another tag: zero)
+__device__ __forceinline__ int sync_count(unsigned long long word, unsigned long long epoch) {
+  return ((word ^ epoch) >> 8) == 0 ? (int)(word & 0xffu) : 0;
+}
+// One more arrival on a sync word; returns the count before it.  Lock-free: an attempt fails only because another
+// arrival succeeded, and a word sees at most a few dozen arrivals per launch.
+__device__ __forceinline__ int sync_arrive(unsigned long long* word, unsigned long long epoch) {
+  unsigned long long old = *reinterpret_cast<volatile unsigned long long*>(word);
+  for (;;) {
+    const unsigned long long cur = ((old ^ epoch) >> 8) == 0 ? old : epoch;
+    const unsigned long long seen = atomicCAS(word, old, cur + 1);
+    if (seen == old) return (int)(cur & 0xffu);
+    old = seen;
+  }
 }
 // orders this thread's generic-proxy observations before its later async-proxy (TMA) accesses
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
@@ -380,11 +401,12 @@ __device__ __forceinline__ float gate_at(const RowGate& g, int j) {
 }
 
 // Bounded acquire-wait until *word >= target.
-__device__ __forceinline__ bool wait_word(const int* word, int target, volatile int* abort_flag) {
-  if (ld_acquire(word) >= target) return true;
+__device__ __forceinline__ bool wait_word(const unsigned long long* word, unsigned long long epoch, int target,
+                                          volatile int* abort_flag) {
+  if (sync_count(ld_acquire(word), epoch) >= target) return true;
   const unsigned long long t0 = global_timer();
   for (uint32_t spins = 1;; ++spins) {
-    if (ld_acquire(word) >= target) return true;
+    if (sync_count(ld_acquire(word), epoch) >= target) return true;
     __nanosleep(64);
     if ((spins & 63u) == 0) {
       if (*abort_flag) return false;
@@ -407,6 +429,10 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
   using L = SmemLayout;
   constexpr uint32_t kTmemCols = kMaxTileW;
 
+  // Programmatic dependent launch: the next launch of this stream may place its CTAs as soon as this grid's CTAs
+  // leave their SMs; it waits below, after its set-up, until this grid has completed and its writes are visible.
+  // (Both instructions do nothing in a launch made without the attribute.)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;     // swizzled tiles need 1024-byte alignment
@@ -457,6 +483,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
   cluster_sync();                                   // the peer's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // nothing before this line reads or writes global memory
 
   int sh_begin = 0;                                 // first shrink item of this pair
   for (int g = 0; g < pair; ++g) sh_begin += pl.sh_count[g];
@@ -495,7 +522,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
           const bool phase1 = b >= item.n_blk0;
           if (phase1 && b == item.n_blk0) {
             // H' of this CTA's row tile must have been published by whoever finished its shrink
-            if (lane == 0 && step_ok) step_ok = wait_word(p.flags + m_tile * pl.n_proj + item.proj, 1, abort_flag);
+            if (lane == 0 && step_ok) step_ok = wait_word(p.flags + m_tile * pl.n_proj + item.proj, p.epoch, 1, abort_flag);
             fence_proxy_async();
           }
           if (!__all_sync(0xffffffffu, step_ok)) { ok = false; break; }
@@ -683,10 +710,10 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
         }
         __threadfence();                             // this thread's partial, device-wide
         epilogue_barrier();
-        int* counter = p.sk_counters + item.tile * 2 + rank;
+        unsigned long long* counter = p.sk_counters + item.tile * 2 + rank;
         if (epi_tid == 0) {
-          atomicAdd(counter, 1);
-          *epi_go = wait_word(counter, pl.split_k, abort_flag) ? 1 : 0;
+          sync_arrive(counter, p.epoch);
+          *epi_go = wait_word(counter, p.epoch, pl.split_k, abort_flag) ? 1 : 0;
         }
         epilogue_barrier();
         if (*epi_go == 0) break;
@@ -783,10 +810,10 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
       __threadfence();                               // this thread's H' / partial stores, device-wide
       epilogue_barrier();
       if (direct) {
-        if (epi_tid == 0 && !p.withhold_publish) st_release(p.flags + sync_idx, 1);
+        if (epi_tid == 0 && !p.withhold_publish) st_release(p.flags + sync_idx, p.epoch | 1ull);
         continue;
       }
-      if (epi_tid == 0) *epi_last = (atomicAdd(p.counters + sync_idx, 1) == pl.shrink_splits - 1);
+      if (epi_tid == 0) *epi_last = (sync_arrive(p.counters + sync_idx, p.epoch) == pl.shrink_splits - 1);
       epilogue_barrier();
       if (*epi_last == 0) continue;
       // this CTA completed its projection's share of the row tile: sum the partials, gate, publish H'
@@ -812,7 +839,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
       }
       __threadfence();
       epilogue_barrier();
-      if (epi_tid == 0 && !p.withhold_publish) st_release(p.flags + sync_idx, 1);
+      if (epi_tid == 0 && !p.withhold_publish) st_release(p.flags + sync_idx, p.epoch | 1ull);
     }
   }
 
@@ -969,7 +996,7 @@ Plan search_plan(int T, int d_in, int n_proj, const int* d_out, int R, int pairs
       if (want > pl.nkb0) break;
       const int per = ceil_div(pl.nkb0, want), splits = ceil_div(pl.nkb0, per);
       const size_t RT = (size_t)n_proj * R;
-      const size_t scratch = (size_t)T * RT * 2 + (size_t)splits * pl.n_m_pairs * 2 * BM * RT * 4 + 4096 + 16 * (size_t)pl.n_m_pairs * n_proj;
+      const size_t scratch = (size_t)T * RT * 2 + (size_t)splits * pl.n_m_pairs * 2 * BM * RT * 4 + 4096 + 32 * (size_t)pl.n_m_pairs * n_proj;
       if (scratch_limit > 0 && splits > 1 && scratch > scratch_limit) continue;
       // measured: a shrink K block costs about 1.3x its staged bytes (narrow MMAs), an item ~4 us of fixed cost
       const long long cs = (long long)per * (16 + 8 * boxes_for(R / 2)) * 13 / 10 + 250;
@@ -1124,11 +1151,24 @@ int max_pairs() {
   return n;
 }
 
+// Launch epochs: 56 bits, starting from a per-process random value so that stale words of another process do not
+// match either; a word of arbitrary memory matches a given launch with probability 2^-56.
+unsigned long long next_epoch() {
+  static std::atomic<unsigned long long> counter{[]() {
+    std::random_device rd;
+    return ((unsigned long long)rd() << 32) ^ (unsigned long long)rd() ^
+           (unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count();
+  }()};
+  unsigned long long e;
+  do { e = counter.fetch_add(1, std::memory_order_relaxed) & ((1ull << 56) - 1); } while (e == 0);
+  return e << 8;
+}
+
 // process-wide test hook state (cwl_debug_set)
 unsigned long long g_wait_limit_ns = kWaitLimitNs;
 int g_withhold_publish = 0;
 
-struct ApplyWorkspace { __nv_bfloat16* Hg; float* partial; float* sk_partial; int* sync; size_t sync_bytes; };
+struct ApplyWorkspace { __nv_bfloat16* Hg; float* partial; float* sk_partial; unsigned long long* sync; size_t sync_bytes; };
 
 // Carves the workspace for a plan.
 size_t carve_apply(ApplyWorkspace& w, char* base, const Plan& pl, int T, int R) {
@@ -1143,9 +1183,9 @@ size_t carve_apply(ApplyWorkspace& w, char* base, const Plan& pl, int T, int R) 
   const bool split = pl.split_k > 1;
   const size_t n_tiles = (size_t)pl.n_m_pairs * pl.n_wide;              // split plans have one tile width
   if (split) off = up(off + n_tiles * pl.split_k * 2 * BM * pl.w0 * sizeof(float));
-  w.sync = reinterpret_cast<int*>(base ? base + off : nullptr);
+  w.sync = reinterpret_cast<unsigned long long*>(base ? base + off : nullptr);
   // shrink counters [2 n_m][n_proj], H' flags [2 n_m][n_proj], split-K counters [2 tiles]
-  w.sync_bytes = sizeof(int) * ((size_t)4 * pl.n_m_pairs * pl.n_proj + (split ? 2 * n_tiles : 0));
+  w.sync_bytes = sizeof(unsigned long long) * ((size_t)4 * pl.n_m_pairs * pl.n_proj + (split ? 2 * n_tiles : 0));
   off = up(off + w.sync_bytes);
   return off < 256 ? 256 : off;
 }
@@ -1230,8 +1270,17 @@ cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* pr
   p.wait_limit_ns = g_wait_limit_ns; p.withhold_publish = g_withhold_publish;
   p.plan = pl;
 
-  // the counters and flags are the only words that must start at zero
-  if (adapter || pl.split_k > 1) CWL_CUDA_TRY(cudaMemsetAsync(ws.sync, 0, ws.sync_bytes, stream));
+  // Every launch tags its sync words with a fresh epoch, so words left by earlier launches (or never written) read as
+  // zero and the workspace needs no clearing: a memset between two kernels costs ~5 us of idle GPU.  Only a launch
+  // that is being captured into a CUDA graph is replayed with the same epoch; it records a clearing node instead.
+  p.epoch = next_epoch();
+  cudaStreamCaptureStatus capture = cudaStreamCaptureStatusNone;
+  CWL_CUDA_TRY(cudaStreamIsCapturing(stream, &capture));
+  if (adapter || pl.split_k > 1) {
+    // (the entry point on the library's own scratch array, the one caller with a scratch limit, clears on every call)
+    if (capture != cudaStreamCaptureStatusNone || scratch_limit > 0)
+      CWL_CUDA_TRY(cudaMemsetAsync(ws.sync, 0, ws.sync_bytes, stream));
+  }
 
   static bool configured[64] = {};  // per device; benign race: the attribute call is idempotent
   int dev = 0;
@@ -1240,8 +1289,20 @@ cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* pr
     CWL_CUDA_TRY(cudaFuncSetAttribute(apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout::kTotal));
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
-  apply_kernel<<<2 * pl.pairs, kThreads, SmemLayout::kTotal, stream>>>(maps, p);
-  CWL_CUDA_TRY(cudaGetLastError());
+  // The kernel-to-kernel gap of a stream (~5 us for this cluster launch) is hidden by letting the launch overlap
+  // the tail of whatever kernel precedes it in the stream; the kernel itself waits for that kernel to complete
+  // before it touches global memory.  Captured launches keep the plain stream order.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pl.pairs, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = SmemLayout::kTotal;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = capture == cudaStreamCaptureStatusNone ? 1 : 0;
+  CWL_CUDA_TRY(cudaLaunchKernelEx(&cfg, apply_kernel, maps, p));
   return CWL_OK;
 }
 

@@ -89,7 +89,7 @@ class HotPath:
     # launches per call, for the benchmark's kernel count
     LAUNCHES_SCORE = 1
     LAUNCHES_PARTITION = 5
-    LAUNCHES_APPLY = 1          # one fused kernel (plus a 256-byte memset node that is not counted)
+    LAUNCHES_APPLY = 1          # one fused kernel
     LAUNCHES_APPLY_DENSE = 1
 
     def set_thresholds(self, thresholds) -> None:
@@ -152,7 +152,7 @@ class HotPath:
             self.apply_step(layer=layer)
 
     def capture(self) -> "torch.cuda.CUDAGraph":
-        """Records one step (every launch and the few-hundred-byte memsets of the sync words) into a CUDA graph.
+        """Records one step (every launch; a captured apply also records a memset of its sync words) into a CUDA graph.
         The library allocates nothing and synchronises nothing on this path; run one ordinary step first so that
         tensor-map descriptors, plans and kernel attributes are set up outside the capture."""
         self.step()

@@ -1,7 +1,8 @@
 """Nothing is written outside the outputs and nothing inside them is left unwritten.  Outputs sit in larger
 buffers filled with a sentinel: guard rows after the last row and guard columns between d_out and the leading
 dimension.  Afterwards every guard still holds the sentinel and no output element does.  Covered: whole-tile
-(TMA-store) epilogue with ragged edges, split-K epilogue, grouped launch, per-row gates, score and partition."""
+epilogue with ragged edges, split-K epilogue, grouped launch, per-row gates, score and partition.  The workspace
+is scratch in the full sense: whatever bytes it holds before a call, the outputs are the same."""
 import numpy as np
 import pytest
 import torch
@@ -55,6 +56,30 @@ def test_cwl_apply_stays_inside_its_output(T, d_in, d_out, R):
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     check_guards(buf, T, d_out)
+
+
+@pytest.mark.parametrize("fill", ["ones", "random", "stale"])
+def test_workspace_contents_do_not_matter(fill):
+    """The counters and flags in the workspace are tagged per launch, so nothing has to be cleared: bytes of any
+    kind (all ones, random, or what earlier calls of other shapes left there) give bit-identical outputs."""
+    shapes = [(300, 1024, 336, 64), (130, 2048, 528, 64), (64, 4096, 4096, 64), (700, 512, 1040, 16)]
+    ws_bytes = max(cwl.cwl_apply_workspace_bytes(T, d_in, d_out, R) for T, d_in, d_out, R in shapes)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for rounds in range(2):
+        for T, d_in, d_out, R in shapes:
+            X, (W,), (A,), (B,) = operands(T + 1, T, d_in, [d_out], R)
+            tab = table(T, R)
+            ref = cwl.cwl_apply(X, W, A, B, tab, 8, workspace=torch.zeros(ws_bytes, dtype=torch.uint8, device="cuda"),
+                                status_word=status)
+            if fill == "ones":
+                ws.fill_(255)
+            elif fill == "random":
+                ws.copy_(torch.randint(0, 256, (ws_bytes,), dtype=torch.uint8, device="cuda"))
+            got = cwl.cwl_apply(X, W, A, B, tab, 8, workspace=ws, status_word=status)      # "stale": left as it is
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            assert torch.equal(ref.view(torch.int16), got.view(torch.int16))
 
 
 def test_grouped_and_per_row_calls_stay_inside_their_outputs():
