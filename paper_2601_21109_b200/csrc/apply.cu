@@ -483,10 +483,16 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
   cluster_sync();                                   // the peer's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  asm volatile("griddepcontrol.wait;" ::: "memory");   // nothing before this line reads or writes global memory
-
   int sh_begin = 0;                                 // first shrink item of this pair
   for (int g = 0; g < pair; ++g) sh_begin += pl.sh_count[g];
+  {
+    // Decoding a work item reads only kernel parameters.  Doing it once before waiting for the launch ahead in the
+    // stream takes the constant-cache misses of the plan out of the time between that launch's end and the first load.
+    Item warm;
+    const bool any = get_item(0, pair, sh_begin, p, warm);
+    asm volatile("" ::"r"(warm.wt + warm.kb0 + warm.n_blk0 + warm.n0 + (any ? 1 : 0)));
+  }
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // nothing before this line reads or writes global memory
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)

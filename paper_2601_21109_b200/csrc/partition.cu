@@ -88,6 +88,8 @@ __device__ int64_t block_sum64(int64_t v, int64_t* smem /* >= 32 entries */) {
 // pass 1: per-tile sums of quantised scores
 __global__ void __launch_bounds__(kScanThreads)
 tile_sum_kernel(const float* __restrict__ score, int T, int64_t* __restrict__ tile_sum) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ int64_t red[32];
   const int base = blockIdx.x * kScanTile;
   int64_t s = 0;
@@ -104,6 +106,8 @@ tile_sum_kernel(const float* __restrict__ score, int T, int64_t* __restrict__ ti
 __global__ void __launch_bounds__(kScanThreads)
 prefix_kernel(const float* __restrict__ score, int T, const int64_t* __restrict__ tile_sum,
               int64_t* __restrict__ P) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ int64_t red[32];
   __shared__ int64_t warp_tot[kScanThreads / 32];
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -144,6 +148,8 @@ prefix_kernel(const float* __restrict__ score, int T, const int64_t* __restrict_
 __global__ void __launch_bounds__(256)
 next_cut_kernel(const int64_t* __restrict__ P, const int32_t* __restrict__ cu, int n_seq, int T,
                 Ladder L, int32_t* __restrict__ next_cut) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int warps_per_block = blockDim.x >> 5;
   for (int64_t b64 = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); b64 < T;
@@ -185,6 +191,8 @@ __global__ void __launch_bounds__(kWalkThreads)
 walk_kernel(const int64_t* __restrict__ P, const int32_t* __restrict__ cu, Ladder L,
             const int32_t* __restrict__ next_cut, int32_t* __restrict__ seq_start,
             int32_t* __restrict__ seq_rung0, int32_t* __restrict__ seq_rung, int32_t* __restrict__ count) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ int32_t seg[kWalkSegment];
   __shared__ int s_pos, s_count;
   const int n = blockIdx.x, tid = threadIdx.x;
@@ -243,6 +251,8 @@ __global__ void __launch_bounds__(256)
 emit_kernel(const int32_t* __restrict__ cu, int n_seq, int T, Ladder L,
             const int32_t* __restrict__ seq_start, const int32_t* __restrict__ seq_rung,
             const int32_t* __restrict__ count, cwl_chunk_table table, int32_t* status_word) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ int64_t red[32];
   const int n = blockIdx.x, tid = threadIdx.x;
   int64_t before = 0;
@@ -326,21 +336,23 @@ extern "C" cwl_status cwl_partition(const float* score, const int32_t* cu_seqlen
     L.theta_q[k] = (int64_t)__builtin_floor((double)policy->threshold[k] * 16777216.0);
 
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const bool chained = !stream_is_capturing(stream);   // each kernel waits for the one before it by itself
   if (T > 0) {
     const int n_tiles = (int)ceil_div64(T, kScanTile);
-    tile_sum_kernel<<<n_tiles, kScanThreads, 0, stream>>>(score, T, w.tile_sum);
-    prefix_kernel<<<n_tiles, kScanThreads, 0, stream>>>(score, T, w.tile_sum, w.P);
+    CWL_CUDA_TRY(launch_chained(chained, tile_sum_kernel, dim3(n_tiles), dim3(kScanThreads), 0, stream, score, T, w.tile_sum));
+    CWL_CUDA_TRY(launch_chained(chained, prefix_kernel, dim3(n_tiles), dim3(kScanThreads), 0, stream, score, T, w.tile_sum, w.P));
     const int warps_per_block = 8;
     int64_t blocks = ceil_div64(T, warps_per_block);
     if (blocks > 148 * 64) blocks = 148 * 64;
-    next_cut_kernel<<<(int)blocks, warps_per_block * 32, 0, stream>>>(w.P, cu_seqlens, n_seq, T, L, w.next_cut);
-    walk_kernel<<<n_seq, kWalkThreads, 0, stream>>>(w.P, cu_seqlens, L, w.next_cut, w.seq_start,
-                                                   w.seq_rung0, w.seq_rung, w.count);
+    CWL_CUDA_TRY(launch_chained(chained, next_cut_kernel, dim3((int)blocks), dim3(warps_per_block * 32), 0, stream, w.P,
+                                cu_seqlens, n_seq, T, L, w.next_cut));
+    CWL_CUDA_TRY(launch_chained(chained, walk_kernel, dim3(n_seq), dim3(kWalkThreads), 0, stream, w.P, cu_seqlens, L,
+                                w.next_cut, w.seq_start, w.seq_rung0, w.seq_rung, w.count));
   } else if (n_seq > 0) {
     CWL_CUDA_TRY(cudaMemsetAsync(w.count, 0, sizeof(int32_t) * (size_t)n_seq, stream));
   }
-  emit_kernel<<<n_seq > 0 ? n_seq : 1, 256, 0, stream>>>(cu_seqlens, n_seq, T, L, w.seq_start, w.seq_rung,
-                                                         w.count, table, status_word);
+  CWL_CUDA_TRY(launch_chained(chained && T > 0, emit_kernel, dim3(n_seq > 0 ? n_seq : 1), dim3(256), 0, stream, cu_seqlens,
+                              n_seq, T, L, w.seq_start, w.seq_rung, w.count, table, status_word));
   CWL_CUDA_TRY(cudaGetLastError());
   return CWL_OK;
 }

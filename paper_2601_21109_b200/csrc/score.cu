@@ -67,6 +67,8 @@ template <bool kMixed>
 __global__ void __launch_bounds__(kScoreThreads)
 score_rows_kernel(const float* __restrict__ logits, int64_t ld, int T, int V, float* __restrict__ score,
                   const MixParams mp) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ Triple warp_part[kScoreThreads / 32];
   __shared__ int warp_bad[kScoreThreads / 32];
   __shared__ int seq_start;
@@ -192,9 +194,9 @@ extern "C" cwl_status cwl_score_tokens(const float* logits, int64_t ld_logits, i
   if (ld_logits < V) return CWL_ERR_SHAPE;
   if ((reinterpret_cast<uintptr_t>(logits) & 3u) != 0) return CWL_ERR_SHAPE;
   int grid = T < (1 << 20) ? T : (1 << 20);
-  cwl::score_rows_kernel<false><<<grid, cwl::kScoreThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-      logits, ld_logits, T, V, score, cwl::MixParams{});
-  CWL_CUDA_TRY(cudaGetLastError());
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CWL_CUDA_TRY(cwl::launch_chained(!cwl::stream_is_capturing(st), cwl::score_rows_kernel<false>, dim3(grid),
+                                   dim3(cwl::kScoreThreads), 0, st, logits, ld_logits, T, V, score, cwl::MixParams{}));
   return CWL_OK;
 }
 
@@ -212,8 +214,8 @@ extern "C" cwl_status cwl_score_tokens_mixed(const float* logits, int64_t ld_log
   cwl::MixParams mp{token_ids, cu_seqlens, n_seq, mix->w_entropy, mix->w_novelty, mix->w_prior,
                     mix->ngram, mix->context, mix->prior_span};
   int grid = T < (1 << 20) ? T : (1 << 20);
-  cwl::score_rows_kernel<true><<<grid, cwl::kScoreThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-      logits, ld_logits, T, V, score, mp);
-  CWL_CUDA_TRY(cudaGetLastError());
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CWL_CUDA_TRY(cwl::launch_chained(!cwl::stream_is_capturing(st), cwl::score_rows_kernel<true>, dim3(grid),
+                                   dim3(cwl::kScoreThreads), 0, st, logits, ld_logits, T, V, score, mp));
   return CWL_OK;
 }

@@ -52,6 +52,8 @@ __global__ void __launch_bounds__(kStreamThreads)
 stream_step_kernel(const float* __restrict__ score, const int32_t* __restrict__ active, int n_seq,
                    const __grid_constant__ StreamLadder L, int32_t* __restrict__ state, int32_t* __restrict__ ring,
                    cwl_row_gate* __restrict__ gates) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int n = blockIdx.x * kStreamThreads + threadIdx.x;
   if (n >= n_seq) return;
   cwl_row_gate g;
@@ -157,9 +159,9 @@ extern "C" cwl_status cwl_stream_step(const float* score, const int32_t* active,
   for (int k = 0; k < CWL_MAX_RUNGS - 1; ++k)
     L.theta_q[k] = k + 1 < policy->n_rungs ? (int64_t)__builtin_floor((double)policy->threshold[k] * 16777216.0) : 0;
   int32_t* words = static_cast<int32_t*>(state);
-  cwl::stream_step_kernel<<<cwl::ceil_div(n_seq, cwl::kStreamThreads), cwl::kStreamThreads, 0,
-                            static_cast<cudaStream_t>(stream)>>>(score, active, n_seq, L, words,
-                                                                 words + (size_t)cwl::kStateWords * n_seq, gates);
-  CWL_CUDA_TRY(cudaGetLastError());
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CWL_CUDA_TRY(cwl::launch_chained(!cwl::stream_is_capturing(st), cwl::stream_step_kernel,
+                                   dim3(cwl::ceil_div(n_seq, cwl::kStreamThreads)), dim3(cwl::kStreamThreads), 0, st, score,
+                                   active, n_seq, L, words, words + (size_t)cwl::kStateWords * n_seq, gates));
   return CWL_OK;
 }

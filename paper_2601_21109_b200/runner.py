@@ -103,11 +103,12 @@ class HotPath:
         cwl.cwl_partition(self.score, self.cu_seqlens, self.cpolicy, table=self.table, workspace=self.part_ws,
                           status_word=self.status)
 
-    # projections that read the same activation go out as one grouped launch: q + k + v and gate + up.  Their
+    # projections that read the same activation go out as one grouped launch where that is measured to pay: their
     # tiles and shrink items are dealt to the CTA pairs together, which fills the last wave of tiles better than
-    # separate calls (measured: a few per cent at T = 2048, about 9 % at T = 8192).
-    GROUPS = (("q", "k", "v"), ("gate", "up"))
-    GROUP_MIN_T = 512           # below this a call is decode-sized: separate calls, whose K loop is split
+    # separate calls.  gate + up (2 x 11008 columns) gain from T = 512 on; q + k + v break even at T = 2048 and
+    # gain 9 % at T = 8192.  Below GROUP_MIN_T a call is decode-sized: separate calls, whose K loop is split.
+    GROUPS = ((("q", "k", "v"), 4096), (("gate", "up"), 512))    # (members, smallest T at which they are grouped)
+    GROUP_MIN_T = 512
 
     def launch_groups(self, layer: int = 0) -> List[List[DeviceProjection]]:
         projs = self.layers[layer]
@@ -118,7 +119,8 @@ class HotPath:
         for p in projs:
             if p.name in used:
                 continue
-            members = next((g for g in self.GROUPS if p.name in g and all(n in by_name for n in g)), (p.name,))
+            members = next((g for g, min_t in self.GROUPS
+                            if p.name in g and self.T >= min_t and all(n in by_name for n in g)), (p.name,))
             out.append([by_name[n] for n in members])
             used.update(members)
         return out
