@@ -17,7 +17,12 @@
  *     wait that ran out) are OR-ed as (1 << status) into *status_word (DEV int32, may be NULL);
  *     the caller zeroes it.  The library never traps, prints or exits.
  *   - Calls on distinct streams may run concurrently as long as they use distinct workspaces.
- *   - The library allocates no device memory in these calls; scratch comes from `workspace`.
+ *   - The library allocates no device memory in these calls; scratch comes from `workspace`,
+ *     whose contents never have to be initialised or cleared by the caller.
+ *   - Kernels are launched so that their set-up may overlap the end of the kernel ahead of them
+ *     in the stream; each waits for that kernel to complete before it reads or writes global
+ *     memory, so stream order holds for every buffer.  Launches recorded by a stream capture use
+ *     plain stream order.
  */
 #ifndef CWL_H
 #define CWL_H
