@@ -18,6 +18,7 @@ constexpr int kScanThreads = 256;
 constexpr int kScanItems = 8;
 constexpr int kScanTile = kScanThreads * kScanItems;  // scores per block in passes 1 and 2
 constexpr int kWalkThreads = 256;
+constexpr int kCutUnroll = 4;         // candidate cuts per lane and round in pass 3
 constexpr int kWalkSegment = 8192;                    // next_cut entries staged per shared-memory segment
 
 struct Ladder {
@@ -102,7 +103,9 @@ tile_sum_kernel(const float* __restrict__ score, int T, int64_t* __restrict__ ti
   if (threadIdx.x == 0) tile_sum[blockIdx.x] = s;
 }
 
-// pass 2: exclusive prefix sums.  Each block adds up the tiles before it, then scans its own.
+// pass 2: exclusive prefix sums.  Each block adds up the tiles before it, then scans its own.  With tile_sum == NULL
+// (a few tiles only: pass 1 is not worth a launch) it adds up the scores before its tile itself; the sums are
+// integers, so the result is the same bit for bit.
 __global__ void __launch_bounds__(kScanThreads)
 prefix_kernel(const float* __restrict__ score, int T, const int64_t* __restrict__ tile_sum,
               int64_t* __restrict__ P) {
@@ -112,7 +115,11 @@ prefix_kernel(const float* __restrict__ score, int T, const int64_t* __restrict_
   __shared__ int64_t warp_tot[kScanThreads / 32];
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   int64_t before = 0;
-  for (int i = tid; i < (int)blockIdx.x; i += kScanThreads) before += tile_sum[i];
+  if (tile_sum != nullptr) {
+    for (int i = tid; i < (int)blockIdx.x; i += kScanThreads) before += tile_sum[i];
+  } else {
+    for (int t = tid; t < (int)blockIdx.x * kScanTile; t += kScanThreads) before += quantise(score[t]);
+  }
   before = block_sum64(before, red);
 
   // thread-contiguous items: thread tid owns [base + tid*kScanItems, +kScanItems)
@@ -167,19 +174,28 @@ next_cut_kernel(const int64_t* __restrict__ P, const int32_t* __restrict__ cu, i
       const int first = b + L.min_len;
       const int last = min(E - L.min_len, b + L.max_len);  // the candidate at b + max_len always stops
       const int64_t Pb = P[b];
-      for (int base = first; base <= last; base += 32) {
-        const int e = base + lane;
-        bool stop = false;
-        if (e <= last) {
-          if (e - b >= L.max_len) {
-            stop = true;
-          } else {
-            const int64_t Pe = P[e];
-            stop = rung_of(Pe - Pb, e - b, L) != rung_of(P[e + L.min_len] - Pe, L.min_len, L);
+      // kCutUnroll x 32 candidates per round, all their loads in flight together (a round is a chain of dependent
+      // L2 accesses, and most chunks close within the first hundred candidates)
+      for (int base = first; base <= last && cut == E; base += 32 * kCutUnroll) {
+        bool stop[kCutUnroll];
+#pragma unroll
+        for (int u = 0; u < kCutUnroll; ++u) {
+          const int e = base + u * 32 + lane;
+          stop[u] = false;
+          if (e <= last) {
+            if (e - b >= L.max_len) {
+              stop[u] = true;
+            } else {
+              const int64_t Pe = P[e];
+              stop[u] = rung_of(Pe - Pb, e - b, L) != rung_of(P[e + L.min_len] - Pe, L.min_len, L);
+            }
           }
         }
-        const unsigned m = __ballot_sync(0xffffffffu, stop);
-        if (m) { cut = base + __ffs(m) - 1; break; }
+#pragma unroll
+        for (int u = 0; u < kCutUnroll; ++u) {
+          const unsigned m = __ballot_sync(0xffffffffu, stop[u]);
+          if (m != 0 && cut == E) cut = base + u * 32 + __ffs(m) - 1;
+        }
       }
     }
     if (lane == 0) next_cut[b] = cut;
@@ -190,7 +206,8 @@ next_cut_kernel(const int64_t* __restrict__ P, const int32_t* __restrict__ cu, i
 __global__ void __launch_bounds__(kWalkThreads)
 walk_kernel(const int64_t* __restrict__ P, const int32_t* __restrict__ cu, Ladder L,
             const int32_t* __restrict__ next_cut, int32_t* __restrict__ seq_start,
-            int32_t* __restrict__ seq_rung0, int32_t* __restrict__ seq_rung, int32_t* __restrict__ count) {
+            int32_t* __restrict__ seq_rung0, int32_t* __restrict__ seq_rung, int32_t* __restrict__ count,
+            bool emit_here, int T, cwl_chunk_table table, int32_t* status_word) {
   pdl_launch_dependents();
   pdl_wait();
   __shared__ int32_t seg[kWalkSegment];
@@ -226,12 +243,11 @@ walk_kernel(const int64_t* __restrict__ P, const int32_t* __restrict__ cu, Ladde
     seq_rung0[S + c] = r;
     seq_rung[S + c] = r;
   }
-  if (L.hi_budget < 0 || L.n_rungs < 2) return;
   __syncthreads();
   // budget on high-capacity regions: a top-rung chunk keeps its rung only if fewer than
   // hi_budget top-rung chunks of this sequence have a larger mean (earlier chunk wins ties)
   const int top = L.n_rungs - 1;
-  for (int c = tid; c < C; c += kWalkThreads) {
+  for (int c = tid; c < C && L.hi_budget >= 0 && L.n_rungs >= 2; c += kWalkThreads) {
     if (seq_rung0[S + c] != top) continue;
     const int bc = seq_start[S + c], ec = (c + 1 < C) ? seq_start[S + c + 1] : E;
     const int64_t sum_c = P[ec] - P[bc], len_c = ec - bc;
@@ -243,6 +259,27 @@ walk_kernel(const int64_t* __restrict__ P, const int32_t* __restrict__ cu, Ladde
       if (lhs > rhs || (lhs == rhs && d < c)) ++better;
     }
     if (better >= L.hi_budget) seq_rung[S + c] = top - 1;
+  }
+  if (!emit_here) return;
+  // a single sequence: this block is the only one, and writes the caller's table itself (pass 5 is not launched)
+  __syncthreads();
+  const bool fits = C <= table.capacity;
+  for (int c = tid; c < C && fits; c += kWalkThreads) {
+    const int r = seq_rung[S + c];
+    table.offsets[c] = seq_start[S + c];
+    table.rung[c] = r;
+    table.rank[c] = L.rung_rank[r];
+    table.scale[c] = L.rung_scale[r];
+    table.flags[c] = (c == 0) ? 1 : 0;
+  }
+  if (tid == 0) {
+    if (fits) {
+      table.offsets[C] = T;
+      *table.n_chunks = C;
+    } else {
+      *table.n_chunks = 0;
+      flag_status(status_word, CWL_ERR_CAPACITY);
+    }
   }
 }
 
@@ -337,22 +374,27 @@ extern "C" cwl_status cwl_partition(const float* score, const int32_t* cu_seqlen
 
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   const bool chained = !stream_is_capturing(stream);   // each kernel waits for the one before it by itself
+  bool emitted = false;
   if (T > 0) {
     const int n_tiles = (int)ceil_div64(T, kScanTile);
-    CWL_CUDA_TRY(launch_chained(chained, tile_sum_kernel, dim3(n_tiles), dim3(kScanThreads), 0, stream, score, T, w.tile_sum));
-    CWL_CUDA_TRY(launch_chained(chained, prefix_kernel, dim3(n_tiles), dim3(kScanThreads), 0, stream, score, T, w.tile_sum, w.P));
+    const bool few_tiles = n_tiles <= 32;                // then pass 2 adds up the scores before its tile itself
+    if (!few_tiles)
+      CWL_CUDA_TRY(launch_chained(chained, tile_sum_kernel, dim3(n_tiles), dim3(kScanThreads), 0, stream, score, T, w.tile_sum));
+    CWL_CUDA_TRY(launch_chained(chained, prefix_kernel, dim3(n_tiles), dim3(kScanThreads), 0, stream, score, T,
+                                few_tiles ? (const int64_t*)nullptr : (const int64_t*)w.tile_sum, w.P));
     const int warps_per_block = 8;
     int64_t blocks = ceil_div64(T, warps_per_block);
     if (blocks > 148 * 64) blocks = 148 * 64;
     CWL_CUDA_TRY(launch_chained(chained, next_cut_kernel, dim3((int)blocks), dim3(warps_per_block * 32), 0, stream, w.P,
                                 cu_seqlens, n_seq, T, L, w.next_cut));
+    emitted = n_seq == 1;                                // one sequence: pass 4 writes the table too
     CWL_CUDA_TRY(launch_chained(chained, walk_kernel, dim3(n_seq), dim3(kWalkThreads), 0, stream, w.P, cu_seqlens, L,
-                                w.next_cut, w.seq_start, w.seq_rung0, w.seq_rung, w.count));
+                                w.next_cut, w.seq_start, w.seq_rung0, w.seq_rung, w.count, emitted, T, table, status_word));
   } else if (n_seq > 0) {
     CWL_CUDA_TRY(cudaMemsetAsync(w.count, 0, sizeof(int32_t) * (size_t)n_seq, stream));
   }
-  CWL_CUDA_TRY(launch_chained(chained && T > 0, emit_kernel, dim3(n_seq > 0 ? n_seq : 1), dim3(256), 0, stream, cu_seqlens,
-                              n_seq, T, L, w.seq_start, w.seq_rung, w.count, table, status_word));
-  CWL_CUDA_TRY(cudaGetLastError());
+  if (!emitted)
+    CWL_CUDA_TRY(launch_chained(chained && T > 0, emit_kernel, dim3(n_seq > 0 ? n_seq : 1), dim3(256), 0, stream, cu_seqlens,
+                                n_seq, T, L, w.seq_start, w.seq_rung, w.count, table, status_word));
   return CWL_OK;
 }

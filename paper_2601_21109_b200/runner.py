@@ -88,7 +88,7 @@ class HotPath:
 
     # launches per call, for the benchmark's kernel count
     LAUNCHES_SCORE = 1
-    LAUNCHES_PARTITION = 5
+    LAUNCHES_PARTITION = 5      # tile sums, prefix, next cut, walk, emit; fewer for small inputs (below)
     LAUNCHES_APPLY = 1          # one fused kernel
     LAUNCHES_APPLY_DENSE = 1
 
@@ -169,7 +169,9 @@ class HotPath:
         if self.logits is not None:
             n += self.LAUNCHES_SCORE
         if not self.fixed_table:
-            n += self.LAUNCHES_PARTITION
+            # up to 32 scan tiles of 2048 scores the tile-sum pass is folded into the prefix pass, and a single
+            # sequence has its table written by the walk pass
+            n += self.LAUNCHES_PARTITION - (1 if self.T <= 32 * 2048 else 0) - (1 if self.n_seq == 1 else 0)
         return n * len(self.layers) + (1 if self.streaming else 0)
 
 

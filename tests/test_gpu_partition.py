@@ -82,6 +82,18 @@ def test_long_sequence_crosses_walk_segments():
     compare(s, np.array([0, T], np.int32), pol)
 
 
+@pytest.mark.parametrize("cu", [[0, 150000], [0, 70001, 70001, 149000, 150000]])
+def test_more_than_32_scan_tiles(cu):
+    """Above 65536 tokens the prefix sums take two passes (tile sums first); below, one.  Both sizes, with one
+    sequence (the walk pass writes the table) and with several (the emit pass does), give the oracle's table."""
+    rng = np.random.default_rng(78)
+    T = cu[-1]
+    s = (np.repeat(rng.random(T // 40 + 1), 40)[:T] + rng.normal(0, 0.03, T)).clip(0, 1).astype(np.float32)
+    pol = wl.Policy.ladder([8, 16, 32, 64], 32.0, [0.25, 0.5, 0.75], min_len=16, window=8, hi_budget=7)
+    compare(s, np.array(cu, np.int32), pol)
+    compare(s[:3000], np.array([0, 1200, 3000], np.int32), pol)
+
+
 def test_many_one_token_sequences():
     T = 300
     s = np.random.default_rng(3).random(T).astype(np.float32)
