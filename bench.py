@@ -323,9 +323,9 @@ def run_ours(args):
     # ---- end to end: pinned host inputs in, results out, every step ----------------------------
     # (the library's HostPipeline: uploads, kernels and downloads of neighbouring steps overlap on three streams)
     e2e_value, e2e_serial, e2e_steps, h2d, d2h = None, None, 0, 0, 0
-    if not args.lean and not streaming:
+    if not args.lean:
         from paper_2601_21109_b200.runner import HostPipeline
-        pipe = HostPipeline(w, n_layers=n_layers, grouped=not args.no_group, first=hp)
+        pipe = HostPipeline(w, n_layers=n_layers, grouped=not args.no_group, first=hp, streaming=streaming)
         h2d, d2h = pipe.h2d_bytes, pipe.d2h_bytes
         e2e_steps = max(4, min(args.steps, 20))
         pipe.run(2)
@@ -345,6 +345,8 @@ def run_ours(args):
                 hp.X[d].copy_(x, non_blocking=True)
             if pipe.host_logits is not None:
                 hp.logits.copy_(pipe.host_logits, non_blocking=True)
+            if pipe.host_score is not None:
+                hp.score.copy_(pipe.host_score, non_blocking=True)
             hp.step()
             for p, y in zip(hp.projs, host_out):
                 y.copy_(p.Y, non_blocking=True)

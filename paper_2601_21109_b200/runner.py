@@ -184,17 +184,21 @@ class HostPipeline:
     slowest of the three instead of their sum.  Weights are shared by the slots."""
 
     def __init__(self, w: Workload, n_layers: int = 1, grouped: bool = True, device: str = "cuda",
-                 first: Optional[HotPath] = None):
-        a = first if first is not None else HotPath(w, device, n_layers=n_layers, grouped=grouped)
-        b = HotPath(w, device, n_layers=n_layers, grouped=grouped, share_weights=a)
+                 first: Optional[HotPath] = None, streaming: bool = False):
+        a = first if first is not None else HotPath(w, device, n_layers=n_layers, grouped=grouped, streaming=streaming)
+        b = HotPath(w, device, n_layers=n_layers, grouped=grouped, streaming=streaming, share_weights=a)
         b.set_thresholds(a.policy.thresholds) if not a.fixed_table and a.logits is not None else None
         self.slots = [a, b]
         self.host_X = {d: x.cpu().pin_memory() for d, x in a.X.items()}
         self.host_logits = a.logits.cpu().pin_memory() if a.logits is not None else None
+        # decode through the scheduler: each slot is its own batch of sequences, and a step's input is one new score
+        # per sequence beside the activations
+        self.host_score = a.score.cpu().pin_memory() if streaming else None
         self.host_Y = [[torch.empty(p.Y.shape, dtype=p.Y.dtype).pin_memory() for p in s.projs] for s in self.slots]
         self.s_in, self.s_run, self.s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
         self.h2d_bytes = sum(x.numel() * x.element_size() for x in self.host_X.values()) + \
-            (self.host_logits.numel() * 4 if self.host_logits is not None else 0)
+            (self.host_logits.numel() * 4 if self.host_logits is not None else 0) + \
+            (self.host_score.numel() * 4 if self.host_score is not None else 0)
         self.d2h_bytes = sum(y.numel() * y.element_size() for y in self.host_Y[0])
 
     def run(self, steps: int):
@@ -213,6 +217,8 @@ class HostPipeline:
                     slot.X[d].copy_(x, non_blocking=True)
                 if self.host_logits is not None:
                     slot.logits.copy_(self.host_logits, non_blocking=True)
+                if self.host_score is not None:
+                    slot.score.copy_(self.host_score, non_blocking=True)
                 uploaded[k] = torch.cuda.Event(); uploaded[k].record(self.s_in)
             with torch.cuda.stream(self.s_run):
                 self.s_run.wait_event(uploaded[k])

@@ -54,3 +54,23 @@ def test_a_captured_step_replays_to_the_same_outputs():
     assert int(hp.status.item()) == 0
     for p, ref in zip(hp.projs, want):
         assert torch.equal(p.Y.view(torch.int16), ref.view(torch.int16))
+
+
+def test_pipelined_decode_through_the_scheduler():
+    """Decode slots advance their own scheduler state: after n pipelined steps a slot's outputs equal those of a
+    plain runner stepped as often as that slot was (slot 0: steps 0, 2, 4; slot 1: steps 1, 3)."""
+    w = wl.config4(T=48)
+    w.policy = wl.Policy.ladder([8, 16, 32, 64], 32.0, [0.25, 0.5, 0.75], min_len=4, window=2)
+    w.score = np.random.default_rng(11).uniform(0, 1, w.T).astype(np.float32)
+    pipe = HostPipeline(w, streaming=True)
+    pipe.run(5)
+    torch.cuda.synchronize()
+    for k, n_steps in ((0, 3), (1, 2)):
+        plain = HotPath(w, streaming=True)
+        for _ in range(n_steps):
+            plain.step()
+        torch.cuda.synchronize()
+        assert int(plain.status.item()) == 0 and int(pipe.slots[k].status.item()) == 0
+        for got, p in zip(pipe.host_Y[k], plain.projs):
+            assert torch.equal(got.view(torch.int16), p.Y.cpu().view(torch.int16))
+    assert pipe.h2d_bytes == 48 * (4096 + 11008) * 2 + 48 * 4
