@@ -424,6 +424,10 @@ struct SmemLayout {
 static_assert(BM * sizeof(RowGate) <= SmemLayout::kOutBytes, "row gates must fit the staging area");
 static_assert(SmemLayout::kTotal <= 227 * 1024, "shared memory budget");
 
+// Two instantiations: kSplitK = false for plans whose tiles keep their whole K loop (the epilogue stores whole
+// tiles), kSplitK = true for plans that split every tile's K loop over several pairs (the epilogue hands partial
+// accumulators over).  A launch runs exactly one of the two epilogues, so neither carries the other's code.
+template <bool kSplitK>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ ApplyParams p) {
   using L = SmemLayout;
@@ -623,7 +627,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
       const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16);
       const int n_chunks = (item.wt + 31) >> 5;
 
-      if (item.kind == ITEM_PROJECT && pl.split_k == 1) {
+      if (!kSplitK && item.kind == ITEM_PROJECT) {
         // ---- whole tile: accumulator -> bf16 -> swizzled staging buffer (a lane holds a row) -> read back so that
         // a warp instruction stores four whole 128-byte row segments ----
         const uint32_t obuf = out_bufs + (uint32_t)(warp - 2) * kOutBufBytes;
@@ -687,7 +691,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
         continue;
       }
 
-      if (item.kind == ITEM_PROJECT) {
+      if (kSplitK && item.kind == ITEM_PROJECT) {
         // ---- split-K item: every contributor owns a share of the tile's columns.  It stores the OTHER columns of
         // its fp32 accumulator (layout [column group of 4][128 rows][4]: a warp's store and the owner's loads are
         // contiguous), waits until all partials of the tile are in, and adds the others' partials of its own
@@ -1145,8 +1149,11 @@ int max_pairs() {
     attr.id = cudaLaunchAttributeClusterDimension;
     attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
     cfg.attrs = &attr; cfg.numAttrs = 1;
-    if (cudaFuncSetAttribute(apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout::kTotal) != cudaSuccess ||
-        cudaOccupancyMaxActiveClusters(&v, apply_kernel, &cfg) != cudaSuccess || v <= 0) {
+    int v2 = 0;
+    if (cudaFuncSetAttribute(apply_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout::kTotal) != cudaSuccess ||
+        cudaFuncSetAttribute(apply_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout::kTotal) != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&v, apply_kernel<false>, &cfg) != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&v2, apply_kernel<true>, &cfg) != cudaSuccess || (v = v < v2 ? v : v2) <= 0) {
       cudaGetLastError();
       v = sms > 0 ? sms / 2 : kPairsPlanned;
     }
@@ -1292,7 +1299,8 @@ cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* pr
   int dev = 0;
   CWL_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64 || !configured[dev]) {
-    CWL_CUDA_TRY(cudaFuncSetAttribute(apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout::kTotal));
+    CWL_CUDA_TRY(cudaFuncSetAttribute(apply_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout::kTotal));
+    CWL_CUDA_TRY(cudaFuncSetAttribute(apply_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout::kTotal));
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
   // The kernel-to-kernel gap of a stream (~5 us for this cluster launch) is hidden by letting the launch overlap
@@ -1308,7 +1316,8 @@ cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* pr
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = capture == cudaStreamCaptureStatusNone ? 1 : 0;
-  CWL_CUDA_TRY(cudaLaunchKernelEx(&cfg, apply_kernel, maps, p));
+  if (pl.split_k > 1) CWL_CUDA_TRY(cudaLaunchKernelEx(&cfg, apply_kernel<true>, maps, p));
+  else CWL_CUDA_TRY(cudaLaunchKernelEx(&cfg, apply_kernel<false>, maps, p));
   return CWL_OK;
 }
 

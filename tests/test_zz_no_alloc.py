@@ -4,6 +4,8 @@ memory (its scratch is a fixed array inside the library).  Collected last on pur
 Checked through the C ABI against the ordinary cwl_apply on the same inputs, on two calls in a row
 with different shapes and tables, so that whatever the first call leaves in the shared scratch must
 not leak into the second."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -38,6 +40,7 @@ def test_matches_cwl_apply_on_two_calls_in_a_row():
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     for (X, W, A, B, tab, window), want in zip(cases, expected):
         Y = torch.empty(X.shape[0], W.shape[1], dtype=torch.bfloat16, device="cuda")
+        gc.collect()                                              # no garbage of earlier tests is freed during the call
         before = torch.cuda.memory_allocated()
         cwl.cwl_apply_noalloc(X, W, A, B, tab, window, Y, status_word=status)
         assert torch.cuda.memory_allocated() == before        # the call itself took nothing from the pool
