@@ -167,6 +167,11 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(map), "r"(leader_bar), "r"(x), "r"(y) : "memory");
 }
+// contiguous global -> shared copy (16-byte aligned, a multiple of 16 bytes) counted on an mbarrier of this CTA
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
@@ -417,7 +422,7 @@ __device__ __forceinline__ bool wait_word(const unsigned long long* word, unsign
 
 struct SmemLayout {
   static constexpr int kOutBytes = kEpiWarps * kOutBufBytes;   // also holds the row gates of a shrink finaliser
-  static constexpr int kBarBytes = (2 * kMaxStages + 2) * 8;
+  static constexpr int kBarBytes = (2 * kMaxStages + 3) * 8;
   static constexpr int kMiscBytes = 32;              // TMEM base, abort flag, epilogue broadcast words
   static constexpr int kTotal = kRingBytes + kOutBytes + kBarBytes + kMiscBytes + 1024;  // + alignment slack
 };
@@ -447,6 +452,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
   auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
   const uint32_t acc_full_bar = bars + 8u * (2 * kMaxStages);
   const uint32_t acc_empty_bar = bars + 8u * (2 * kMaxStages + 1);
+  const uint32_t fix_bar = bars + 8u * (2 * kMaxStages + 2);   // split-K: the others' partial sums have landed
   uint8_t* misc = base_ptr + kRingBytes + L::kOutBytes + L::kBarBytes;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
@@ -468,6 +474,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     mbar_init(acc_full_bar, 1);
     mbar_init(acc_empty_bar, 2 * kEpiWarps);
+    mbar_init(fix_bar, 1);
     *abort_flag = 0;
     *reinterpret_cast<volatile unsigned long long*>(abort_flag + 3) = p.wait_limit_ns;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -721,12 +728,36 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
         __threadfence();                             // this thread's partial, device-wide
         epilogue_barrier();
         unsigned long long* counter = p.sk_counters + item.tile * 2 + rank;
+        // The others' partial sums of this CTA's share are one contiguous run per contributor: where they fit the
+        // (now idle) operand ring beside the staged rows, bulk copies bring them in at once instead of a chain of
+        // dependent loads per thread.
+        const uint32_t seg_bytes = (uint32_t)(c_hi - c_lo) * (BM * 4);          // one contributor's run
+        const uint32_t land = ((uint32_t)(BM * pitch) + 1023u) & ~1023u;        // offset of the landing zone in the ring
+        const bool landed = c_hi > c_lo && land + (uint32_t)(pl.split_k - 1) * seg_bytes <= (uint32_t)kRingBytes;
         if (epi_tid == 0) {
           sync_arrive(counter, p.epoch);
-          *epi_go = wait_word(counter, p.epoch, pl.split_k, abort_flag) ? 1 : 0;
+          const bool in = wait_word(counter, p.epoch, pl.split_k, abort_flag);
+          if (in && landed) {
+            fence_proxy_async();                     // the partials were written with ordinary stores
+            mbar_expect_tx(fix_bar, (uint32_t)(pl.split_k - 1) * seg_bytes);
+            int slot = 0;
+            for (int s = 0; s < pl.split_k; ++s) {
+              if (s == item.split) continue;
+              bulk_load(base + land + slot * seg_bytes, tile_base + s * split_stride + (int64_t)(c_lo >> 2) * (BM * 4), seg_bytes, fix_bar);
+              ++slot;
+            }
+          }
+          *epi_go = in ? 1 : 0;
         }
         epilogue_barrier();
         if (*epi_go == 0) break;
+        if (landed) {
+          mbar_wait(fix_bar, 0, abort_flag);         // a failure is recorded in abort_flag
+          epilogue_barrier();
+          if (epi_tid == 0) *epi_go = (*abort_flag == 0);
+          epilogue_barrier();
+          if (*epi_go == 0) break;
+        }
         __threadfence();
 #pragma unroll 1
         for (int cc = (c_lo >> 5) + ((((c_lo >> 5) & 1) != chalf) ? 1 : 0); cc * 32 < c_hi; cc += 2) {
@@ -736,17 +767,34 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
           float acc[32];
 #pragma unroll
           for (int j = 0; j < 32; ++j) acc[j] = __uint_as_float(v[j]);
-          const float* src0 = tile_base + ((int64_t)(cc * 8) * BM + row_in_tile) * 4;
-#pragma unroll 2
-          for (int s = 0; s < pl.split_k; ++s) {
-            if (s == item.split) continue;
-            const float* src = src0 + s * split_stride;
+          if (landed) {
+            // landing zone: [contributor][column group of 4 from c_lo][128 rows][4]
+            const uint32_t l0 = base + land + (uint32_t)(((cc * 8 - (c_lo >> 2)) * BM + row_in_tile) * 16);
+#pragma unroll 1
+            for (int slot = 0; slot < pl.split_k - 1; ++slot) {
 #pragma unroll
-            for (int q4 = 0; q4 < 8; ++q4) {
-              const int col = cc * 32 + q4 * 4;
-              if (col >= c_lo && col < c_hi) {
-                const float4 x = __ldcg(reinterpret_cast<const float4*>(src + q4 * BM * 4));
-                acc[q4 * 4 + 0] += x.x; acc[q4 * 4 + 1] += x.y; acc[q4 * 4 + 2] += x.z; acc[q4 * 4 + 3] += x.w;
+              for (int q4 = 0; q4 < 8; ++q4) {
+                const int col = cc * 32 + q4 * 4;
+                if (col >= c_lo && col < c_hi) {
+                  const uint4 x = ld_shared_v4(l0 + slot * seg_bytes + q4 * (BM * 16));
+                  acc[q4 * 4 + 0] += __uint_as_float(x.x); acc[q4 * 4 + 1] += __uint_as_float(x.y);
+                  acc[q4 * 4 + 2] += __uint_as_float(x.z); acc[q4 * 4 + 3] += __uint_as_float(x.w);
+                }
+              }
+            }
+          } else {
+            const float* src0 = tile_base + ((int64_t)(cc * 8) * BM + row_in_tile) * 4;
+#pragma unroll 2
+            for (int s = 0; s < pl.split_k; ++s) {
+              if (s == item.split) continue;
+              const float* src = src0 + s * split_stride;
+#pragma unroll
+              for (int q4 = 0; q4 < 8; ++q4) {
+                const int col = cc * 32 + q4 * 4;
+                if (col >= c_lo && col < c_hi) {
+                  const float4 x = __ldcg(reinterpret_cast<const float4*>(src + q4 * BM * 4));
+                  acc[q4 * 4 + 0] += x.x; acc[q4 * 4 + 1] += x.y; acc[q4 * 4 + 2] += x.z; acc[q4 * 4 + 3] += x.w;
+                }
               }
             }
           }
