@@ -725,8 +725,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
                   make_uint4(v[q4 * 4 + 0], v[q4 * 4 + 1], v[q4 * 4 + 2], v[q4 * 4 + 3]);
           }
         }
-        __threadfence();                             // this thread's partial, device-wide
-        epilogue_barrier();
+        epilogue_barrier();                          // every thread's partial stores precede thread 0's release below
         unsigned long long* counter = p.sk_counters + item.tile * 2 + rank;
         // The others' partial sums of this CTA's share are one contiguous run per contributor: where they fit the
         // (now idle) operand ring beside the staged rows, bulk copies bring them in at once instead of a chain of
@@ -735,8 +734,9 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
         const uint32_t land = ((uint32_t)(BM * pitch) + 1023u) & ~1023u;        // offset of the landing zone in the ring
         const bool landed = c_hi > c_lo && land + (uint32_t)(pl.split_k - 1) * seg_bytes <= (uint32_t)kRingBytes;
         if (epi_tid == 0) {
+          __threadfence();                           // device-wide release of the CTA's partial (cumulative over the barrier)
           sync_arrive(counter, p.epoch);
-          const bool in = wait_word(counter, p.epoch, pl.split_k, abort_flag);
+          bool in = wait_word(counter, p.epoch, pl.split_k, abort_flag);
           if (in && landed) {
             fence_proxy_async();                     // the partials were written with ordinary stores
             mbar_expect_tx(fix_bar, (uint32_t)(pl.split_k - 1) * seg_bytes);
@@ -746,19 +746,14 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
               bulk_load(base + land + slot * seg_bytes, tile_base + s * split_stride + (int64_t)(c_lo >> 2) * (BM * 4), seg_bytes, fix_bar);
               ++slot;
             }
+            in = mbar_wait(fix_bar, 0, abort_flag);  // bounded; a failure is recorded in abort_flag
           }
           *epi_go = in ? 1 : 0;
         }
         epilogue_barrier();
         if (*epi_go == 0) break;
-        if (landed) {
-          mbar_wait(fix_bar, 0, abort_flag);         // a failure is recorded in abort_flag
-          epilogue_barrier();
-          if (epi_tid == 0) *epi_go = (*abort_flag == 0);
-          epilogue_barrier();
-          if (*epi_go == 0) break;
-        }
-        __threadfence();
+        if (landed) mbar_wait(fix_bar, 0, abort_flag);   // completed already: every thread observes the copies itself
+        else __threadfence();
 #pragma unroll 1
         for (int cc = (c_lo >> 5) + ((((c_lo >> 5) & 1) != chalf) ? 1 : 0); cc * 32 < c_hi; cc += 2) {
           uint32_t v[32];
