@@ -171,8 +171,8 @@ cwl_status cwl_apply_grouped(const void* X, int64_t ldx, const cwl_projection* p
                              int32_t T, int32_t d_in, int32_t R, cwl_chunk_table table, int32_t window,
                              void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream);
 
-/* Decode-time scheduler (Sec. III-A "streaming and cached", III-B "grouped online", III-F "state cached across
- * steps"): every step brings one new token per sequence.  The paper names the constraints only; the rule here is
+/* Decode-time scheduler (Sec. III-A, III-B, III-F: scores arrive as tokens stream in, tokens are grouped as they
+ * arrive, and the scheduler keeps its state from step to step): every step brings one new token per sequence.  The paper names the constraints only; the rule here is
  * causal.  Per sequence the state holds the open chunk's length and the rung it was opened on, the rung of the chunk
  * before it, and the quantised scores of the last min_len tokens.  A new token first enters that trailing window;
  * the first token of a sequence opens the first chunk on the window's rung; later, a chunk of at least min_len

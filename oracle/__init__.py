@@ -220,7 +220,7 @@ ROW_GATE_DTYPE = np.dtype([("rank_in", np.int32), ("rank_out", np.int32), ("scal
 
 
 class Stream:
-    """Decode-time scheduler of ONE sequence (Sec. III-B "grouped online", state cached across steps)."""
+    """Decode-time scheduler of ONE sequence (Sec. III-B: tokens are grouped as they arrive; the state is kept from step to step)."""
 
     def __init__(self, ranks, scales, thresholds, min_len, max_len, window, hi_budget=-1):
         self.policy = _policy_struct(ranks, scales, thresholds, min_len, max_len, window, hi_budget)

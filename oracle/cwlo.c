@@ -69,7 +69,7 @@ int cwlo_score_tokens(const float* logits, int64_t ld, int32_t T, int32_t V, dou
 }
 
 /* ---------------------------------------------------------------------------------------------
- * Sec. III-B "average-complexity threshold": chunk means are compared in fixed point so that
+ * Sec. III-B (a chunk is judged by its mean complexity against thresholds): chunk means are compared in fixed point so that
  * the partition is a function of the fp32 score array alone, independent of summation order.
  * ------------------------------------------------------------------------------------------- */
 int64_t cwlo_quantise(float s) {
@@ -278,8 +278,8 @@ int cwlo_apply(const uint16_t* X, int64_t ldx, const uint16_t* W, int64_t ldw,
 }
 
 /* ---------------------------------------------------------------------------------------------
- * Decode-time scheduler (Sec. III-A "streaming and cached", III-B "grouped online", III-F "the
- * scheduler's state is cached across steps").  The paper names the constraints only; the rule is
+ * Decode-time scheduler (Sec. III-A, III-B, III-F: scores arrive as tokens stream in, tokens are
+ * grouped as they arrive, and the scheduler keeps its state from step to step).  The paper names the constraints only; the rule is
  * this build's causal reading: a token may open a new chunk only on what has been seen so far.
  *
  * Per sequence: the open chunk's length and the rung it was opened on (a chunk's configuration is

@@ -1,5 +1,6 @@
-// cwl_stream_*: decode-time scheduler.  One new token per sequence and step (Sec. III-A "streaming and
-// cached", Sec. III-B "grouped online", Sec. III-F "the scheduler's state is cached across steps").
+// cwl_stream_*: decode-time scheduler.  One new token per sequence and step (Sec. III-A: complexity is
+// estimated as tokens stream in; Sec. III-B: tokens are grouped as they arrive; Sec. III-F: the scheduler keeps its
+// state from step to step).
 //
 // State per sequence, struct of arrays on the device so that thread n's accesses coalesce with its
 // neighbours': tokens seen, length and rung of the open chunk, rung of the chunk before it, top-rung

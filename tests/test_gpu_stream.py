@@ -1,5 +1,5 @@
-"""GPU parity of the decode-time scheduler (cwl_stream_*, Sec. III-B "grouped online" with state cached across
-steps) and of the per-row adapted projection cwl_apply_rows, against the oracle, through the C ABI.
+"""GPU parity of the decode-time scheduler (cwl_stream_*, Sec. III-B: tokens grouped as they arrive, state kept from step
+to step) and of the per-row adapted projection cwl_apply_rows, against the oracle, through the C ABI.
 Gates are integer decisions plus copied scales and an fp32 quotient: compared bit by bit."""
 import numpy as np
 import pytest
