@@ -103,6 +103,18 @@ def test_static_lora_and_decode_tables_small():
     run_case(T, 128, 128, 64, w4.table, 0, seed=21)
 
 
+def test_split_k_with_partials_too_large_to_land():
+    """Decode-sized rows against a large projection: 512-wide tiles whose K loop is split 3-way.  The two other
+    contributors' partial sums of a CTA's share (2 x 88 KB) do not fit the operand ring beside the staged rows,
+    so the hand-over reads them from global memory instead of landing them by bulk copies."""
+    T, d_in, d_out = 8, 11008, 11008
+    plan = cwl.cwl_apply_plan(T, d_in, d_out, 64)
+    assert plan["split_k"] == 3 and plan["wide_width"] == 512
+    w4 = wl.config4(T=T)
+    run_case(T, d_in, d_out, 64, w4.table, 0, seed=22)
+    run_case(T, d_in, d_out, 64, None, 0, seed=23, adapter=False)
+
+
 def test_argument_errors():
     X = torch.zeros(8, 64, dtype=torch.bfloat16, device="cuda")
     W = torch.zeros(64, 64, dtype=torch.bfloat16, device="cuda")
