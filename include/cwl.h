@@ -210,7 +210,8 @@ cwl_status cwl_apply_rows(const void* X, int64_t ldx, const void* W, int64_t ldw
                           const cwl_row_gate* gates, void* Y, int64_t ldy,
                           void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream);
 
-/* Offline construction of the rank ladder (Sec. III-C: "obtained once by SVD of the adapter matrix"): re-factorises a
+/* Offline construction of the rank ladder (Sec. III-C: the ladder comes from a one-off singular value decomposition
+ * of the trained adapter): re-factorises a
  * trained adapter so that every prefix of the stored factors is the best adapter of its rank,
  *   A B = U diag(sigma) V^T,  A_out = U diag(sigma) [d_in, R],  B_out = V^T [R, d_out],  sigma descending,
  * by two one-sided Jacobi passes in fp64 (no d_in x d_out product, no Gram matrix).  Not on the timed path: the call

@@ -1496,6 +1496,16 @@ extern "C" cwl_status cwl_apply_noalloc(const void* X, int64_t ldx, const void* 
                                         void* Y, int64_t ldy, int32_t* status_word, void* stream) {
   if (T < 0 || d_in < 1 || d_out < 1 || R < 0) return CWL_ERR_INVALID_ARG;
   const bool adapter = (A != nullptr && B != nullptr && R > 0);
+  {
+    // the same argument checks, in the same order, as cwl_apply makes: a bad shape is reported as such, not as a
+    // scratch problem
+    cwl_projection q;
+    q.W = W; q.ldw = ldw; q.A = adapter ? A : nullptr; q.lda = lda; q.B = adapter ? B : nullptr; q.ldb = ldb;
+    q.Y = Y; q.ldy = ldy; q.d_out = d_out;
+    bool with_adapter = false;
+    const cwl_status chk = cwl::check_group(X, ldx, &q, 1, T, d_in, R, table, nullptr, window, with_adapter);
+    if (chk != CWL_OK) return chk;
+  }
   if (adapter && T > 0 && cwl_apply_noalloc_scratch_need(T, d_in, d_out, R) > (size_t)CWL_NOALLOC_SCRATCH_BYTES)
     return CWL_ERR_WORKSPACE;  // the problem needs more scratch than the built-in array holds
   void* scratch = nullptr;

@@ -33,18 +33,60 @@ def y_to_f64(Y: torch.Tensor) -> np.ndarray:
     return bf16_bits_to_f32(bits).astype(np.float64)
 
 
-def check_output(y_gpu: np.ndarray, y_ref: np.ndarray):
-    """Relative Frobenius <= 1e-2; every entry within 3e-2, or within one bf16 ulp of the rounded
-    reference (half an ulp of bf16 alone exceeds 3e-2 once |y| >= 8).  Returns the figures."""
+def bf16_ulp(x: np.ndarray) -> np.ndarray:
+    """Spacing of bf16 numbers in the binade of x: 2^(floor(log2 |x|) - 7) (8 significand bits)."""
+    _, e = np.frexp(np.abs(x))                       # |x| = m 2^e, m in [0.5, 1): floor(log2 |x|) = e - 1
+    return np.ldexp(1.0, np.maximum(e - 1, -126) - 7)
+
+
+# figures of every check_output call of the session, printed at its end (tests/conftest.py)
+REPORT = []
+
+
+def check_output(y_gpu: np.ndarray, y_ref: np.ndarray, label: str = "", max_saved_frac: float = 1e-3):
+    """Relative Frobenius <= 1e-2; every entry within 3e-2, or within ONE bf16 ulp (the spacing of bf16 in the
+    binade of the correctly rounded reference) of that rounded reference: half an ulp of bf16 alone exceeds
+    3e-2 once |y| >= 8, so a perfect kernel can miss 3e-2 by output rounding.  Entries that pass by the ulp
+    clause only must have |ref| >= 4 (below that one ulp is within 3e-2 anyway) and stay a small fraction of
+    the output; their count and the strict max-abs error are returned and recorded."""
     diff = np.abs(y_gpu - y_ref)
     rel_fro = float(np.linalg.norm(y_gpu - y_ref) / max(np.linalg.norm(y_ref), 1e-30))
     ref_bf16 = bf16_bits_to_f32(f32_to_bf16_bits(y_ref.astype(np.float32))).astype(np.float64)
-    ulp = np.maximum(np.abs(ref_bf16), 2.0 ** -126) * 2.0 ** -7
-    within_ulp = np.abs(y_gpu - ref_bf16) <= ulp
+    within_ulp = np.abs(y_gpu - ref_bf16) <= bf16_ulp(ref_bf16)
     bad = (diff > 3e-2) & ~within_ulp
+    saved = (diff > 3e-2) & within_ulp
+    res = dict(label=label, rel_fro=rel_fro, max_abs=float(diff.max()) if diff.size else 0.0,
+               saved_by_ulp=int(saved.sum()), entries=int(diff.size),
+               min_abs_ref_saved=float(np.abs(ref_bf16[saved]).min()) if saved.any() else None)
+    REPORT.append(res)
     assert rel_fro <= 1e-2, f"relative Frobenius error {rel_fro:.3e}"
     assert not bad.any(), f"{int(bad.sum())} entries off by more than 3e-2 and one bf16 ulp; max abs {diff.max():.3e}"
-    return dict(rel_fro=rel_fro, max_abs=float(diff.max()), saved_by_ulp=int(((diff > 3e-2) & within_ulp).sum()))
+    assert not saved.any() or res["min_abs_ref_saved"] >= 4.0, "the ulp clause decided an entry with |ref| < 4"
+    assert res["saved_by_ulp"] <= max(4, max_saved_frac * diff.size), \
+        f"{res['saved_by_ulp']} of {diff.size} entries pass by the ulp clause only"
+    return res
+
+
+SCORE_REPORT = []
+
+
+def check_scores(s_gpu: np.ndarray, s_ref: np.ndarray, label: str = ""):
+    """fp32 scores within 1e-5 relative, the denominator floored at 1e-2 (a relative bound on a quantity that tends
+    to 0 is ill-posed); NaN exactly where the reference has NaN.  The strict relative error (no floor; entries whose
+    reference is exactly 0 count by their absolute error) is recorded beside it."""
+    s_gpu = np.asarray(s_gpu, np.float64); s_ref = np.asarray(s_ref, np.float64)
+    nan = np.isnan(s_ref)
+    assert np.array_equal(np.isnan(s_gpu), nan)
+    g, r = s_gpu[~nan], s_ref[~nan]
+    if g.size == 0:
+        return 0.0
+    err = np.abs(g - r)
+    floored = err / np.maximum(np.abs(r), 1e-2)
+    strict = np.where(r != 0.0, err / np.where(r != 0.0, np.abs(r), 1.0), err)
+    i = int(np.argmax(strict))
+    SCORE_REPORT.append(dict(label=label, floored=float(floored.max()), strict=float(strict.max()), at=float(abs(r[i]))))
+    assert floored.max() <= 1e-5, f"max relative error {floored.max():.3e}"
+    return float(floored.max())
 
 
 def status_ok(status_word: torch.Tensor):
