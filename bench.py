@@ -1,25 +1,32 @@
 #!/usr/bin/env python
 """Benchmark of the ChunkWise-LoRA hot path on B200.
 
-One step = one pass of the whole hot path over one batch of the LLaMA-7B-shaped prefill
-configuration (T = 2048 tokens): token scoring from fp32 logits [T, 32000], adaptive partition and
-rank selection, then the adapted projection for all seven projections (q, k, v, o, gate, up, down)
+Headline workload (default): the 32-layer LLaMA-7B-shaped projection stack, 4 sequences x 4096 tokens.  One step =
+one pass of the whole hot path over that batch: per layer, token scoring from fp32 logits [16384, 32000], adaptive
+partition and rank selection, then the adapted projection for all seven projections (q, k, v, o, gate, up, down)
 with R = 64.  Prints ONE JSON line: metric, value (whole-job tokens/s), ms_per_step, config, clocks, e2e (host
-buffers in and out every step), gpu_launches, roofline (dominant kernel against the measured peaks) and
-cpu_baseline (the fp64 oracle timed on the host cores).
+buffers in and out every step), gpu_launches, roofline (dominant kernel against the measured peaks), cpu_baseline
+(the fp64 oracle timed on the host cores) and, at one GPU, a `configs` block with the same measurement on the other
+workloads (single-sequence prefill, packed ragged prefill, decode with a fixed table, decode through the scheduler).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload cfg2|cfg3|cfg4|cfg4_stream|cfg5|cfg1] [--layers L] [--no-group] [--lean]
+                    [--workload cfg5|cfg2|cfg3|cfg4|cfg4_stream|cfg1] [--layers L] [--min-seconds S]
+                    [--no-configs] [--no-group] [--no-prefetch] [--lean]
 
-N > 1 runs N independent replicas (one process per GPU, launched with torch.distributed.run); the
-path has no exchange step, so there is no data-path collective: only the timing barrier and the
-max-over-ranks reduction of the timed region.
+Every timed region lasts at least --min-seconds of device time: the block of K steps is repeated (`inner_repeats`)
+until it does, and ms_per_step is the mean over all K x repeats steps (median and min per block are beside it).
+
+N > 1 runs N independent replicas (one process per GPU; without a launcher the script starts its own ranks through
+torch.distributed.run); the path has no exchange step, so there is no data-path collective: only the timing barrier
+and the max-over-ranks reduction of the timed region.
 """
 from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -33,6 +40,8 @@ sys.path.insert(0, ROOT)
 
 METRIC = "adapted_projection_tokens_per_s"
 UNIT = "tokens/s"
+SUB_CONFIGS = ("cfg2", "cfg3", "cfg4", "cfg4_stream")
+DECODE_WEIGHT_SETS = 4      # decode steps rotate over this many weight sets so that no step finds its weights in L2
 
 
 # ------------------------------------------------------------------------------------ helpers
@@ -156,7 +165,40 @@ def make_workload(name: str):
     raise SystemExit(f"unknown workload {name}")
 
 
-# ----------------------------------------------------------------------------- reference arm
+def layers_of(name: str, args) -> int:
+    """Weight sets resident on the device: the stack's layers, or the sets a decode run rotates over."""
+    if name == "cfg5":
+        return args.layers
+    return DECODE_WEIGHT_SETS if name in ("cfg4", "cfg4_stream") else 1
+
+
+def config_dict(name: str, w, n_layers: int, world: int, grouped: bool) -> dict:
+    """What was run, from the workload alone (the same for both arms)."""
+    decode = name in ("cfg4", "cfg4_stream")
+    streaming = name == "cfg4_stream"
+    has_logits, fixed = w.logits is not None, w.table is not None
+    parts = (["scheduler step"] if streaming else []) + (["score"] if has_logits else []) + \
+        ([] if (fixed or streaming) else ["partition"]) + [f"{len(w.projections)} adapted projections"]
+    stack = n_layers if name == "cfg5" else 1
+    steps_include = (f"{stack} layers x (" if stack > 1 else "(") + " + ".join(parts) + ")"
+    step_bytes = stack * (sum(2 * p.d_in * p.d_out for p in w.projections) +
+                          (int(w.logits.size) * 4 if has_logits else 0))
+    if decode:
+        l2 = (f"steps rotate over {n_layers} distinct weight sets ({n_layers * step_bytes / 1e6:.0f} MB), so every "
+              f"step streams its {step_bytes / 1e6:.0f} MB of weights from HBM; no flush needed")
+    elif step_bytes > 126e6:
+        l2 = f"inputs larger than L2 ({step_bytes / 1e6:.0f} MB of weights and logits read per step); no flush needed"
+    else:
+        l2 = (f"inputs smaller than L2 ({step_bytes / 1e6:.1f} MB per step), not flushed: activations and outputs "
+              f"stream, the one weight matrix is reused by every row tile anyway")
+    return {"workload": w.name, "T": int(w.T), "R": int(w.R),
+            "projections": [f"{p.name}:{p.d_in}x{p.d_out}" for p in w.projections],
+            "ladder": list(w.policy.ranks), "window": int(w.policy.window), "min_len": int(w.policy.min_len),
+            "layers": stack, "n_seq": int(len(w.cu_seqlens) - 1), "steps_include": steps_include, "l2": l2,
+            "grouped_launches": bool(grouped), "parallelism": "replicas only" if world > 1 else "single GPU"}
+
+
+# ----------------------------------------------------------------------------- the oracle, timed
 def oracle_sample(w, n_rows: int, n_score_rows: int = 64):
     """Times the fp64 CPU oracle on a bounded sample of the workload; returns (tokens/s, info)."""
     import oracle
@@ -204,24 +246,73 @@ def rows_for_budget(w, seconds: float):
     return int(min(w.T, cores * waves)), t_wave
 
 
+def oracle_full_legs(w2=None) -> dict:
+    """The oracle timed in full where that takes seconds: the small single-projection configuration end to end,
+    on one thread and on all host cores, and the scorer and the chunker on the whole single-sequence prefill
+    inputs (2048 x 32000 logits)."""
+    import oracle
+    from paper_2601_21109_b200 import workloads as wl
+    legs = {}
+    all_cores = oracle.get_threads()
+    w1 = wl.config1()
+    p, pr = w1.policy, w1.projections[0]
+    for label, n in (("one_thread", 1), ("all_cores", all_cores)):
+        oracle.set_threads(n)
+        t0 = time.perf_counter()
+        tab = oracle.partition(w1.score, w1.cu_seqlens, p.ranks, p.scales, p.thresholds, p.min_len, p.max_len, p.window, p.hi_budget)
+        oracle.apply(w1.X[pr.d_in], pr.W, pr.A, pr.B, tab, p.window)
+        dt = time.perf_counter() - t0
+        legs[f"cfg1_full_{label}"] = {"seconds": dt, "tokens_per_s": w1.T / dt, "threads": n,
+                                      "what": "partition + apply, all 256 rows x 1024 columns"}
+    if w2 is None:
+        w2 = wl.config2()
+    p2 = w2.policy
+    for label, n in (("one_thread", 1), ("all_cores", all_cores)):
+        oracle.set_threads(n)
+        t0 = time.perf_counter()
+        s = oracle.score_tokens(w2.logits)
+        dt = time.perf_counter() - t0
+        legs[f"cfg2_score_full_{label}"] = {"seconds": dt, "tokens_per_s": w2.T / dt, "threads": n,
+                                            "what": f"cwlo_score_tokens on logits [{w2.T}, {w2.logits.shape[1]}]"}
+    oracle.set_threads(all_cores)
+    s32 = s.astype(np.float32)
+    ths = np.percentile(s32, [25, 50, 75]).astype(np.float32).tolist()
+    reps = 20
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        oracle.partition(s32, w2.cu_seqlens, p2.ranks, p2.scales, ths, p2.min_len, p2.max_len, p2.window, p2.hi_budget)
+    dt = (time.perf_counter() - t0) / reps
+    legs["cfg2_partition_full"] = {"seconds": dt, "tokens_per_s": w2.T / dt, "threads": 1,
+                                   "what": f"cwlo_partition on all {w2.T} scores (sequential by definition)"}
+    return legs
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     w = make_workload(args.workload)
+    n_layers = layers_of(args.workload, args)
+    stack = n_layers if args.workload == "cfg5" else 1
     budget = 150.0 / (args.steps + args.warmup)         # the whole run ends within a few minutes
     n_rows, _ = rows_for_budget(w, budget)
-    vals = []
+    vals, secs = [], []
     info = {}
     for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
         v, info = oracle_sample(w, n_rows)
         if i >= args.warmup:
-            vals.append(v)
+            vals.append(v / stack)
+            secs.append(time.perf_counter() - t0)
     value = float(np.mean(vals))
+    if stack > 1:
+        info["sample"] += f"; one layer timed, divided by {stack} layers"
+    info["note"] = ("ms_per_step is the wall time of one step's bounded sample; value scales the sample to the whole "
+                    "workload (per-row cost is constant)")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.T / value,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(secs)),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "T": w.T, "R": w.R, "projections": [f"{p.name}:{p.d_in}x{p.d_out}" for p in w.projections]},
+            "config": config_dict(args.workload, w, n_layers, args.gpus, not args.no_group),
             "cpu_baseline": dict(value=value, unit=UNIT, **info),
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -229,12 +320,224 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------- our arm
+def measure(name: str, args, steps: int, warmup: int, world: int, rank: int, local_rank: int, full: bool):
+    """Builds one workload on the device, times it, and returns (result dict, workload)."""
+    import torch
+    from paper_2601_21109_b200 import binding as cwl
+    from paper_2601_21109_b200 import replicas
+    from paper_2601_21109_b200 import workloads as wl
+    from paper_2601_21109_b200.runner import HotPath
+
+    w = make_workload(name)
+    n_layers = layers_of(name, args)
+    stack = n_layers if name == "cfg5" else 1           # layers one step runs through
+    decode = name in ("cfg4", "cfg4_stream")
+    streaming = name == "cfg4_stream"
+    hp = HotPath(w, n_layers=n_layers, grouped=not args.no_group, streaming=streaming, prefetch=not args.no_prefetch)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        replicas.barrier(world)
+
+    def run_step(i: int):
+        # a decode step works on ONE weight set, the next step on the next one; a stack step runs every layer
+        if decode:
+            hp.step(layer=i % n_layers)
+        else:
+            hp.step()
+
+    # thresholds of the rule-based percentile mapping (Sec. IV-C): quartiles of this batch's scores
+    if hp.logits is not None:
+        hp.score_step()
+        s = hp.score.cpu().numpy()
+        hp.set_thresholds(np.percentile(s, [25, 50, 75]).astype(np.float32).tolist())
+    run_step(0)
+    torch.cuda.synchronize()
+    if int(hp.status.item()) != 0:
+        raise SystemExit(f"device status word {int(hp.status.item()):#x}")
+    table = hp.table.to_host() if not streaming else None
+    proj_dims = [(p.d_in, p.d_out) for p in hp.projs]
+    if table is not None:
+        f_alg, f_exe = table_flops(table, hp.policy.window, hp.T, proj_dims, hp.R)
+    else:   # row gates change every step: count the executed (full-rank) work
+        f_alg = f_exe = sum(2 * hp.T * di * do + 2 * hp.T * hp.R * (di + do) for di, do in proj_dims)
+    f_alg, f_exe = f_alg * stack, f_exe * stack
+
+    # ---- device-resident timing: blocks of `steps` steps, no event inside a block ---------------
+    for i in range(warmup):
+        run_step(i)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record(stream)
+    for i in range(steps):
+        run_step(i)
+    b.record(stream)
+    torch.cuda.synchronize()
+    block_ms = max(a.elapsed_time(b), 1e-3)
+    repeats = max(1, int(math.ceil(args.min_seconds * 1e3 / block_ms)))
+    if world > 1:
+        repeats = int(replicas.max_over_ranks(float(repeats), world))     # every rank runs the same count
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(repeats + 1)]
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    barrier()
+    t_wall0 = time.time()
+    marks[0].record(stream)
+    for r in range(repeats):
+        for i in range(steps):
+            run_step(r * steps + i)
+        marks[r + 1].record(stream)
+    barrier()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    ms_total = replicas.max_over_ranks(marks[0].elapsed_time(marks[-1]), world)
+    block_list = [marks[r].elapsed_time(marks[r + 1]) / steps for r in range(repeats)]
+    if int(hp.status.item()) != 0:
+        raise SystemExit(f"device status word {int(hp.status.item()):#x}")
+    n_steps = steps * repeats
+    value = replicas.job_throughput(hp.T, n_steps, world, ms_total)
+    ms_per_step = ms_total / n_steps
+
+    # ---- the apply launches alone, inside whole steps (second pass: the headline span above has no inner event) ----
+    if decode and not streaming:
+        apply_ms = ms_per_step                  # the step IS its apply launches
+    else:
+        n2 = max(steps, min(n_steps, int(math.ceil(0.5e3 / max(ms_per_step, 1e-3)))))
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n2 * stack)]
+        for i in range(n2):
+            if streaming:
+                hp.stream_state.step(hp.score)
+            for layer in range(stack):
+                L = (i % n_layers) if decode else layer
+                if hp.logits is not None:
+                    hp.score_step()
+                if not hp.fixed_table and not streaming:
+                    hp.partition_step()
+                ev[i * stack + layer][0].record(stream)
+                hp.apply_step(layer=L)
+                ev[i * stack + layer][1].record(stream)
+        torch.cuda.synchronize()
+        apply_ms = sum(x.elapsed_time(y) for x, y in ev) / n2
+
+    # ---- comparison runs through the same kernels: static full-rank LoRA and the dense floor ---
+    static_ms = dense_ms = chunk_only_ms = None
+    if not args.lean:
+        st = wl.static_table(w.cu_seqlens, hp.R, 32.0)
+        static_tab = cwl.DeviceChunkTable.from_host(st["offsets"], st["rank"], st["scale"], st["flags"], st["rung"])
+
+        def time_apply(**kw):
+            est = max(apply_ms, 1e-3)
+            n = max(3, int(math.ceil(0.4e3 / est)))
+            for i in range(3):
+                for layer in range(stack):
+                    hp.apply_step(layer=(i % n_layers) if decode else layer, **kw)
+            x, y = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            x.record(stream)
+            for i in range(n):
+                for layer in range(stack):
+                    hp.apply_step(layer=(i % n_layers) if decode else layer, **kw)
+            y.record(stream)
+            torch.cuda.synchronize()
+            return x.elapsed_time(y) / n
+        chunk_only_ms = time_apply()
+        static_ms = time_apply(table=static_tab)
+        dense_ms = time_apply(dense=True)
+
+    # ---- end to end: pinned host inputs in, results out, every step ----------------------------
+    e2e = None
+    if full and not args.lean:
+        from paper_2601_21109_b200.runner import HostPipeline
+        pipe = HostPipeline(w, n_layers=n_layers, grouped=not args.no_group, first=hp, streaming=streaming)
+        e2e_steps = max(4, min(steps, 20))
+        pipe.run(2)
+        barrier()
+        x, y = pipe.run(e2e_steps)
+        barrier()
+        e2e_ms = replicas.max_over_ranks(x.elapsed_time(y), world)
+        e2e_value = replicas.job_throughput(hp.T, e2e_steps, world, e2e_ms)
+        for slot in pipe.slots:
+            if int(slot.status.item()) != 0:
+                raise SystemExit(f"device status word {int(slot.status.item()):#x}")
+        host_out = pipe.host_Y[0]
+
+        def serial_step():      # the same without overlap (one stream): plain copy - step - copy
+            for d, xx in pipe.host_X.items():
+                hp.X[d].copy_(xx, non_blocking=True)
+            if pipe.host_logits is not None:
+                hp.logits.copy_(pipe.host_logits, non_blocking=True)
+            if pipe.host_score is not None:
+                hp.score.copy_(pipe.host_score, non_blocking=True)
+            hp.step()
+            for p, yy in zip(hp.projs, host_out):
+                yy.copy_(p.Y, non_blocking=True)
+        serial_step()
+        barrier()
+        x, y = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        x.record(stream)
+        for _ in range(max(2, e2e_steps // 2)):
+            serial_step()
+        y.record(stream)
+        barrier()
+        serial = replicas.job_throughput(hp.T, max(2, e2e_steps // 2), world, replicas.max_over_ranks(x.elapsed_time(y), world))
+        e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": pipe.h2d_bytes, "d2h_bytes_per_step": pipe.d2h_bytes,
+               "steps": e2e_steps, "serial_value": serial,
+               "how": "HostPipeline: two device slots, upload / kernels / download of neighbouring steps overlapped on "
+                      "three streams; inputs are copied once per step (a stack step re-scores the same logits in every layer)"}
+        del pipe
+
+    # ---- roofline of the dominant kernel (the projection GEMM inside cwl_apply) -----------------
+    peaks = load_peaks()
+    capped = bool(clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and
+                  clocks["sm_mhz"] < 0.9 * clocks["sm_max_mhz"] and "sw_power_cap" in clocks.get("reasons", []))
+    if decode:
+        bytes_alg = sum(2 * (hp.T * di + di * do + hp.R * (di + do) + hp.T * do) + 2 * hp.T * hp.R * 2 for di, do in proj_dims)
+        achieved = bytes_alg / (apply_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": load_traffic("apply_" + name),
+                "peak_source": f"hbm copy, of {peaks['source']}", "algorithmic_bytes_per_step": bytes_alg,
+                "frac_of_nominal_8000": achieved / 8000.0}
+    else:
+        # the sustained peak when the sampled clocks show the region ran power-capped, the burst one otherwise
+        kind = "bf16_tflops_sustained" if capped else "bf16_tflops"
+        achieved = f_alg / (apply_ms * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks[kind], "unit": "TFLOP/s",
+                "frac": achieved / peaks[kind], "traffic": load_traffic("apply_" + name),
+                "peak_source": f"{kind} ({'power-capped' if capped else 'uncapped'} region by the sampled clocks), of {peaks['source']}",
+                "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
+                "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
+                "executed_tflops": f_exe / (apply_ms * 1e-3) / 1e12, "frac_of_nominal_2250": achieved / 2250.0}
+    roof["kernel"] = ("cwl::apply_kernel (one fused launch per projection or projection group: shrink, gate, base GEMM + "
+                      "expand); achieved = the step's algorithmic FLOPs or bytes over the event-timed span of its apply launches")
+    roof["launch_ms"] = apply_ms
+    roof["sm_mhz_median"] = clocks.get("sm_mhz") if clocks else None
+    if clocks and clocks.get("sm_mhz"):
+        roof["launch_ms_x_mhz"] = apply_ms * clocks["sm_mhz"]
+
+    res = {"value": value, "unit": UNIT, "ms_per_step": ms_per_step, "ms_per_step_median": float(statistics.median(block_list)),
+           "ms_per_step_min": float(min(block_list)), "steps": steps, "inner_repeats": repeats,
+           "timed_region_s": ms_total * 1e-3,
+           "config": dict(config_dict(name, w, n_layers, world, not args.no_group)),
+           "n_chunks": int(table["n_chunks"]) if table is not None else None,
+           "tflops": f_alg * n_steps * world / (ms_total * 1e-3) / 1e12,
+           "apply_ms_per_step": apply_ms, "apply_only_loop_ms": chunk_only_ms,
+           "static_lora_apply_ms": static_ms, "dense_floor_apply_ms": dense_ms,
+           "clocks": clocks, "gpu_launches": hp.launches_per_step(stack) * n_steps, "roofline": roof}
+    if e2e is not None:
+        res["e2e"] = e2e
+    del hp
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    return res, w
+
+
 def run_ours(args):
     import torch
     from paper_2601_21109_b200 import binding as cwl
-    from paper_2601_21109_b200.runner import HotPath
-
     from paper_2601_21109_b200 import replicas
+
     rank, local_rank, world = replicas.world_from_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
@@ -242,194 +545,56 @@ def run_ours(args):
     replicas.init("nccl", local_rank, world)
     cwl.lib()  # fails loudly when libcwl.so is missing
 
-    w = make_workload(args.workload)
-    n_layers = args.layers if args.workload == "cfg5" else 1
-    streaming = args.workload == "cfg4_stream"
-    hp = HotPath(w, n_layers=n_layers, grouped=not args.no_group, streaming=streaming)
-    stream = torch.cuda.current_stream()
+    head, w = measure(args.workload, args, args.steps, args.warmup, world, rank, local_rank, full=True)
 
-    # thresholds of the rule-based percentile mapping (Sec. IV-C): quartiles of this batch's scores
-    if hp.logits is not None:
-        hp.score_step()
-        s = hp.score.cpu().numpy()
-        hp.set_thresholds(np.percentile(s, [25, 50, 75]).astype(np.float32).tolist())
-    hp.step()
-    torch.cuda.synchronize()
-    if int(hp.status.item()) != 0:
-        raise SystemExit(f"device status word {int(hp.status.item()):#x}")
-    table = hp.table.to_host()
-    proj_dims = [(p.d_in, p.d_out) for p in hp.projs]
-    f_alg, f_exe = table_flops(table, hp.policy.window, hp.T, proj_dims, hp.R)
-    f_alg, f_exe = f_alg * n_layers, f_exe * n_layers
-
-    def barrier():
-        replicas.barrier(world)
-
-    # ---- device-resident timing --------------------------------------------------------------
-    for _ in range(args.warmup):
-        hp.step()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-          for _ in range(args.steps * n_layers)]
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.25)
-    barrier()
-    t_wall0 = time.time()
-    e0.record(stream)
-    for i in range(args.steps):
-        if streaming:
-            hp.stream_state.step(hp.score)
-        for layer in range(n_layers):
-            if hp.logits is not None:
-                hp.score_step()
-            if not hp.fixed_table:
-                hp.partition_step()
-            ev[i * n_layers + layer][0].record(stream)
-            hp.apply_step(layer=layer)
-            ev[i * n_layers + layer][1].record(stream)
-    e1.record(stream)
-    barrier()
-    t_wall1 = time.time()
-    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
-    ms_total = e0.elapsed_time(e1)
-    apply_ms = [sum(a.elapsed_time(b) for a, b in ev[i * n_layers:(i + 1) * n_layers]) for i in range(args.steps)]
-    ms_total = replicas.max_over_ranks(ms_total, world)
-    if int(hp.status.item()) != 0:
-        raise SystemExit(f"device status word {int(hp.status.item()):#x}")
-    value = replicas.job_throughput(hp.T, args.steps, world, ms_total)
-
-    # ---- comparison runs through the same kernels: static full-rank LoRA and the dense floor ---
-    from paper_2601_21109_b200 import workloads as wl
-    st = wl.static_table(w.cu_seqlens, hp.R, 32.0)
-    static_tab = cwl.DeviceChunkTable.from_host(st["offsets"], st["rank"], st["scale"], st["flags"], st["rung"])
-
-    def time_apply(**kw):
-        for _ in range(3):
-            hp.apply_step(**kw)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        n = max(3, min(args.steps, 50))
-        a.record(stream)
-        for _ in range(n):
-            for layer in range(n_layers):
-                hp.apply_step(layer=layer, **kw)
-        b.record(stream)
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) / n
-    static_ms = None if args.lean else time_apply(table=static_tab)
-    dense_ms = None if args.lean else time_apply(dense=True)
-
-    # ---- end to end: pinned host inputs in, results out, every step ----------------------------
-    # (the library's HostPipeline: uploads, kernels and downloads of neighbouring steps overlap on three streams)
-    e2e_value, e2e_serial, e2e_steps, h2d, d2h = None, None, 0, 0, 0
-    if not args.lean:
-        from paper_2601_21109_b200.runner import HostPipeline
-        pipe = HostPipeline(w, n_layers=n_layers, grouped=not args.no_group, first=hp, streaming=streaming)
-        h2d, d2h = pipe.h2d_bytes, pipe.d2h_bytes
-        e2e_steps = max(4, min(args.steps, 20))
-        pipe.run(2)
-        barrier()
-        a, b = pipe.run(e2e_steps)
-        barrier()
-        e2e_ms = replicas.max_over_ranks(a.elapsed_time(b), world)
-        e2e_value = replicas.job_throughput(hp.T, e2e_steps, world, e2e_ms)
-        for slot in pipe.slots:
-            if int(slot.status.item()) != 0:
-                raise SystemExit(f"device status word {int(slot.status.item()):#x}")
-        # the same without overlap (one stream): what a caller gets from plain copy - step - copy
-        host_out = pipe.host_Y[0]
-
-        def serial_step():
-            for d, x in pipe.host_X.items():
-                hp.X[d].copy_(x, non_blocking=True)
-            if pipe.host_logits is not None:
-                hp.logits.copy_(pipe.host_logits, non_blocking=True)
-            if pipe.host_score is not None:
-                hp.score.copy_(pipe.host_score, non_blocking=True)
-            hp.step()
-            for p, y in zip(hp.projs, host_out):
-                y.copy_(p.Y, non_blocking=True)
-        serial_step()
-        barrier()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        for _ in range(e2e_steps):
-            serial_step()
-        b.record(stream)
-        barrier()
-        e2e_serial = replicas.job_throughput(hp.T, e2e_steps, world, replicas.max_over_ranks(a.elapsed_time(b), world))
+    configs, w2 = {}, None
+    if world == 1 and not args.lean and not args.no_configs and args.workload == "cfg5":
+        for name in SUB_CONFIGS:
+            k = {"cfg2": 200, "cfg3": 100, "cfg4": 1000, "cfg4_stream": 1000}[name]
+            sub, ws = measure(name, args, k, 5, world, rank, local_rank, full=False)
+            if name == "cfg2":
+                w2 = ws
+            sub["metric"] = METRIC
+            configs[name] = sub
 
     if rank != 0:
         replicas.finish(world)
         return
 
-    # ---- roofline of the dominant kernel (the projection GEMM inside cwl_apply) -----------------
-    peaks = load_peaks()
-    apply_avg_ms = float(np.mean(apply_ms))
-    region_s = ms_total * 1e-3
-    if args.workload in ("cfg4", "cfg4_stream"):
-        bytes_alg = sum(2 * (hp.T * di + di * do + hp.R * (di + do) + hp.T * do) + 2 * hp.T * hp.R * 2 for di, do in proj_dims)
-        achieved = bytes_alg / (apply_avg_ms * 1e-3) / 1e9
-        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": load_traffic("apply_" + args.workload),
-                "peak_source": f"hbm copy, of {peaks['source']}"}
+    stack = head["config"]["layers"]
+    if args.lean or world > 1:
+        cpu = {}
     else:
-        # sustained peak for a long or power-capped region (SM clock pulled well below its maximum), burst otherwise
-        capped = bool(clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and
-                      clocks["sm_mhz"] < 0.85 * clocks["sm_max_mhz"] and "sw_power_cap" in clocks.get("reasons", []))
-        kind = "bf16_tflops_sustained" if (region_s > 1.0 or capped) else "bf16_tflops"
-        achieved = f_alg / (apply_avg_ms * 1e-3) / 1e12
-        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks[kind], "unit": "TFLOP/s",
-                "frac": achieved / peaks[kind], "traffic": load_traffic("apply_" + args.workload),
-                "peak_source": f"{kind}, of {peaks['source']}"}
-    roof["kernel"] = ("cwl::apply_kernel (one fused launch per projection: shrink, gate, base GEMM + expand); achieved = the "
-                      "step's algorithmic FLOPs or bytes over the event-timed span of its apply launches")
-    if roof["bound"] == "tensor":
-        roof["frac_of_burst_peak"] = roof["achieved"] / peaks["bf16_tflops"]
-        roof["frac_of_sustained_peak"] = roof["achieved"] / peaks["bf16_tflops_sustained"]
-    roof["launch_ms"] = apply_avg_ms
-    roof["executed_tflops"] = f_exe / (apply_avg_ms * 1e-3) / 1e12
-    roof["frac_of_nominal_2250"] = (f_alg / (apply_avg_ms * 1e-3) / 1e12) / 2250.0
-
-    parts = (["scheduler step"] if streaming else []) + (["score"] if hp.logits is not None else []) + ([] if hp.fixed_table else ["partition"]) + \
-        [f"{len(hp.projs)} projections in {len(hp.launch_groups())} apply launches"]
-    steps_include = (f"{n_layers} layers x (" if n_layers > 1 else "(") + " + ".join(parts) + ")"
-    step_bytes = n_layers * (sum(2 * p.d_in * p.d_out for p in hp.projs) +
-                             (hp.logits.numel() * 4 if hp.logits is not None else 0))
-    l2_note = (f"inputs larger than L2 ({step_bytes / 1e6:.0f} MB of weights and logits read per step)"
-               if step_bytes > 126e6 else
-               f"inputs smaller than L2 ({step_bytes / 1e6:.1f} MB per step), not flushed: parity-sized workload, not a headline")
-    if args.lean:
-        cpu_val, cpu_info = None, {}
-    else:
-        n_rows, _ = rows_for_budget(w, 12.0)         # about 10-20 s of CPU work
+        n_rows, _ = rows_for_budget(w, 10.0)         # about 10-20 s of CPU work
         cpu_val, cpu_info = oracle_sample(w, n_rows=n_rows)
-        if n_layers > 1:
-            cpu_val /= n_layers
-            cpu_info["sample"] += f"; one layer timed, divided by {n_layers} layers"
+        if stack > 1:
+            cpu_val /= stack
+            cpu_info["sample"] += f"; one layer timed, divided by {stack} layers"
+        cpu = dict(value=cpu_val, unit=UNIT, **cpu_info)
+        cpu["full_runs"] = oracle_full_legs(w2)
 
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": w.name, "T": hp.T, "R": hp.R, "projections": [f"{p.name}:{p.d_in}x{p.d_out}" for p in hp.projs],
-                   "ladder": hp.policy.ranks, "window": hp.policy.window, "min_len": hp.policy.min_len,
-                   "n_chunks": table["n_chunks"], "layers": n_layers, "steps_include": steps_include, "l2": l2_note,
-                   "parallelism": "replicas only" if world > 1 else "single GPU"},
-        "tflops": f_alg * args.steps * world / (ms_total * 1e-3) / 1e12,
-        "apply_ms_per_step": apply_avg_ms,
-        "static_lora_apply_ms": static_ms, "dense_floor_apply_ms": dense_ms,
-        "clocks": clocks,
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
-                "how": "HostPipeline: two device slots, upload / kernels / download of neighbouring steps overlapped on three streams",
-                "serial_value": e2e_serial},
-        "gpu_launches": hp.launches_per_step() * args.steps,
-        "roofline": roof,
-        "cpu_baseline": dict(value=cpu_val, unit=UNIT, **cpu_info),
+        "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": head["ms_per_step"], "ms_per_step_median": head["ms_per_step_median"],
+        "ms_per_step_min": head["ms_per_step_min"], "inner_repeats": head["inner_repeats"],
+        "timed_region_s": head["timed_region_s"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": head["config"], "n_chunks": head["n_chunks"], "tflops": head["tflops"],
+        "apply_ms_per_step": head["apply_ms_per_step"], "apply_only_loop_ms": head["apply_only_loop_ms"],
+        "static_lora_apply_ms": head["static_lora_apply_ms"], "dense_floor_apply_ms": head["dense_floor_apply_ms"],
+        "clocks": head["clocks"], "e2e": head.get("e2e"), "gpu_launches": head["gpu_launches"],
+        "roofline": head["roofline"], "cpu_baseline": cpu,
     }
+    if configs:
+        line["configs"] = configs
     print(json.dumps(line))
     replicas.finish(world)
+
+
+def free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
 
 
 def main():
@@ -438,21 +603,31 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg4_stream", "cfg5"])
+    ap.add_argument("--workload", default="cfg5", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg4_stream", "cfg5"])
     ap.add_argument("--layers", type=int, default=32, help="layers of the cfg5 projection stack (a step runs all of them)")
+    ap.add_argument("--min-seconds", type=float, default=2.0,
+                    help="least device time of a timed region; the block of --steps steps is repeated until it is reached")
+    ap.add_argument("--no-configs", action="store_true", help="headline workload only: no `configs` block")
     ap.add_argument("--no-group", action="store_true",
                     help="one cwl_apply launch per projection instead of grouped launches for q,k,v and gate,up")
+    ap.add_argument("--no-prefetch", action="store_true",
+                    help="decode: do not tell a call which weights the next call streams (no L2 prefetch while it drains)")
     ap.add_argument("--lean", action="store_true",
                     help="timed region only (no comparison runs, end-to-end leg or CPU baseline): for profiler runs")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # no launcher around us: start one rank per GPU ourselves; rank 0 prints the line
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+               "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.run(cmd).returncode)
     if args.impl == "reference":
         args.steps = 2 if args.steps is None else max(1, args.steps)
         args.warmup = 1 if args.warmup is None else max(0, args.warmup)
         run_reference(args)
     else:
-        default_steps = {"cfg5": 5, "cfg3": 100}.get(args.workload, 500)
+        default_steps = {"cfg5": 3, "cfg3": 100, "cfg4": 1000, "cfg4_stream": 1000}.get(args.workload, 200)
         args.steps = default_steps if args.steps is None else max(1, args.steps)
-        args.warmup = max(5 if args.warmup is None else args.warmup, 3)
+        args.warmup = max(3 if args.warmup is None else args.warmup, 3)
         run_ours(args)
 
 

@@ -229,6 +229,19 @@ cwl_status cwl_ladder_build(const void* A, int64_t lda, const void* B, int64_t l
                             float* A_out_f32, float* B_out_f32, float* sigma,
                             void* workspace, size_t workspace_bytes, int32_t* sweeps, void* stream);
 
+/* One-shot hint for the NEXT cwl_apply / cwl_apply_rows / cwl_apply_grouped call made by this host thread: the
+ * region [ptr, ptr + bytes) is what the call AFTER that one will stream -- typically the weight matrix of the
+ * projection that follows (weights and adapter factors are frozen at inference: Sec. III-C).  Once a CTA of the
+ * hinted launch has issued its last operand load, it asks L2 for its slice of the region, so that HBM keeps
+ * working while the launch combines its partial sums and stores its outputs, and while the following launch
+ * sets up; that launch then finds (part of) its weights in L2.  It matters for decode-sized calls, which are
+ * bound by HBM and whose drain is a large share of the launch; at most ~100 MB (less than L2) is useful.
+ *   ptr   DEV, any alignment (whole 128-byte lines inside the region are requested); must stay valid until the
+ *         hinted launch has completed.  The data is only read.  NULL or bytes == 0 withdraws a pending hint.
+ * The hint is consumed by the next call whether or not that call launches anything; it has no effect on results.
+ * Thread-local; no device work is done by this call itself. */
+cwl_status cwl_prefetch_next(const void* ptr, size_t bytes);
+
 /* Test hook for the failure path of cwl_apply and its variants.  Every device-side wait (mbarrier, H' flag, split-K
  * counter) is bounded; when one runs out the CTA raises CWL_ERR_TIMEOUT in *status_word (bit 1 << CWL_ERR_TIMEOUT),
  * drains its copies, frees its tensor memory and returns, so the context stays usable.  This call sets the limit

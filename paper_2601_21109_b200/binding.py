@@ -23,7 +23,7 @@ EXPORTS = ["cwl_status_string", "cwl_version", "cwl_score_tokens", "cwl_score_to
            "cwl_partition", "cwl_apply_workspace_bytes", "cwl_apply", "cwl_apply_grouped_workspace_bytes",
            "cwl_apply_grouped", "cwl_apply_plan", "cwl_stream_state_bytes", "cwl_stream_reset", "cwl_stream_step",
            "cwl_apply_rows", "cwl_ladder_workspace_bytes", "cwl_ladder_build", "cwl_debug_set",
-           "cwl_apply_noalloc_scratch_need", "cwl_apply_noalloc"]
+           "cwl_apply_noalloc_scratch_need", "cwl_apply_noalloc", "cwl_prefetch_next"]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 
 
@@ -130,6 +130,8 @@ def lib():
         L.cwl_ladder_build.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
                                        C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_size_t, C.POINTER(C.c_int32), C.c_void_p]
+        L.cwl_prefetch_next.restype = C.c_int
+        L.cwl_prefetch_next.argtypes = [C.c_void_p, C.c_size_t]
         L.cwl_debug_set.restype = None
         L.cwl_debug_set.argtypes = [C.c_int64, C.c_int32]
         L.cwl_apply_plan.restype = C.c_int
@@ -408,6 +410,15 @@ def cwl_ladder_build(A: torch.Tensor, B: torch.Tensor, want_f32: bool = True,
         _p(out.get("A32")), _p(out.get("B32")), _p(out["sigma"]), _p(ws), ws.numel(), C.byref(sweeps), _stream_ptr(stream)))
     out["sweeps"] = int(sweeps.value)
     return out
+
+
+def cwl_prefetch_next(t: Optional[torch.Tensor]) -> None:
+    """One-shot hint: the next apply call of this thread asks L2, while it drains, for the memory of `t` (the
+    weights the call after it will stream).  None withdraws a pending hint."""
+    if t is None:
+        lib().cwl_prefetch_next(None, 0)
+    else:
+        _check("cwl_prefetch_next", lib().cwl_prefetch_next(_p(t), t.numel() * t.element_size()))
 
 
 def cwl_debug_set(wait_limit_ns: int = 0, withhold_publish: bool = False) -> None:

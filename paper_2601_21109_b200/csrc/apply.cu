@@ -110,6 +110,8 @@ struct ApplyParams {
   cwl_chunk_table table;
   const cwl_row_gate* row_gates;   // when set: one descriptor per row instead of the chunk table
   unsigned long long wait_limit_ns; // limit of every device-side wait
+  const unsigned char* pf_ptr;      // hinted region the NEXT call will stream (its weights), 128-byte aligned; or null
+  unsigned long long pf_bytes;      // its size, a multiple of 128
   int withhold_publish;            // test hook: never publish H', so that the waits on it run out
   int32_t* status_word;
   Plan plan;
@@ -171,6 +173,10 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// asks L2 for a contiguous run of global memory (16-byte aligned, a multiple of 16 bytes); no destination, no completion
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
@@ -554,6 +560,21 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
             tma_load_2d_pair(sb + bi * kBoxBytes, phase1 ? map1 : map0, leader_full, box_x, k);
           }
           if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
+        }
+      }
+      if (ok && p.pf_bytes != 0) {
+        // All of this CTA's loads are issued.  From here to the end of the launch (the last K blocks, the hand-over of
+        // partial sums, the output stores) and through the start of the next launch HBM would sit idle: ask L2 for this
+        // CTA's slice of the region the caller says the next call streams.  Read-only, no completion to wait for.
+        constexpr unsigned long long kPiece = 8192;
+        const unsigned long long n_cta = gridDim.x;
+        unsigned long long slice = (p.pf_bytes + n_cta - 1) / n_cta;
+        slice = (slice + 127ull) & ~127ull;
+        const unsigned long long lo = (unsigned long long)blockIdx.x * slice;
+        const unsigned long long hi = lo + slice < p.pf_bytes ? lo + slice : p.pf_bytes;
+        for (unsigned long long off = lo + (unsigned long long)lane * kPiece; off < hi; off += 32ull * kPiece) {
+          const unsigned long long n = hi - off < kPiece ? hi - off : kPiece;
+          bulk_prefetch_l2(p.pf_ptr + off, (uint32_t)n);
         }
       }
       if (!ok && rank == 0 && lane == 0) {
@@ -1220,6 +1241,10 @@ unsigned long long next_epoch() {
   return e << 8;
 }
 
+// One-shot hint of the calling host thread (cwl_prefetch_next): consumed by its next apply launch.
+struct NextPrefetch { const unsigned char* ptr; unsigned long long bytes; };
+thread_local NextPrefetch t_next_prefetch = {nullptr, 0};
+
 // process-wide test hook state (cwl_debug_set)
 unsigned long long g_wait_limit_ns = kWaitLimitNs;
 int g_withhold_publish = 0;
@@ -1281,6 +1306,9 @@ cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* pr
                             int32_t d_in, int32_t R, cwl_chunk_table table, int32_t window, void* workspace,
                             size_t workspace_bytes, int32_t* status_word, void* stream_, bool allow_split_k,
                             size_t scratch_limit, const cwl_row_gate* row_gates = nullptr) {
+  // the calling thread's one-shot prefetch hint belongs to this call, whatever becomes of it
+  const NextPrefetch hint = t_next_prefetch;
+  t_next_prefetch = {nullptr, 0};
   bool adapter = false;
   const cwl_status chk = check_group(X, ldx, proj, n_proj, T, d_in, R, table, row_gates, window, adapter);
   if (chk != CWL_OK) return chk;
@@ -1325,6 +1353,7 @@ cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* pr
   p.table = table; p.row_gates = row_gates; p.status_word = status_word;
   p.wait_limit_ns = g_wait_limit_ns; p.withhold_publish = g_withhold_publish;
   p.plan = pl;
+  p.pf_ptr = hint.ptr; p.pf_bytes = hint.bytes;
 
   // Every launch tags its sync words with a fresh epoch, so words left by earlier launches (or never written) read as
   // zero and the workspace needs no clearing: a memset between two kernels costs ~5 us of idle GPU.  Only a launch
@@ -1385,6 +1414,16 @@ extern "C" size_t cwl_apply_workspace_bytes(int32_t T, int32_t d_in, int32_t d_o
   cwl::ApplyWorkspace w;
   const cwl::Plan pl = cwl::make_plan(T, d_in, 1, &d_out, R, cwl::max_pairs(), true);
   return cwl::carve_apply(w, nullptr, pl, T, R);
+}
+
+extern "C" cwl_status cwl_prefetch_next(const void* ptr, size_t bytes) {
+  if (ptr == nullptr || bytes == 0) { cwl::t_next_prefetch = {nullptr, 0}; return CWL_OK; }
+  // whole 128-byte lines inside [ptr, ptr + bytes)
+  const uintptr_t lo = (reinterpret_cast<uintptr_t>(ptr) + 127u) & ~(uintptr_t)127u;
+  const uintptr_t hi = (reinterpret_cast<uintptr_t>(ptr) + bytes) & ~(uintptr_t)127u;
+  if (hi <= lo) { cwl::t_next_prefetch = {nullptr, 0}; return CWL_OK; }
+  cwl::t_next_prefetch = {reinterpret_cast<const unsigned char*>(lo), (unsigned long long)(hi - lo)};
+  return CWL_OK;
 }
 
 extern "C" void cwl_debug_set(int64_t wait_limit_ns, int32_t withhold_publish) {

@@ -36,8 +36,10 @@ class HotPath:
     """Device-resident state of one layer's adapted projections plus the scheduler in front."""
 
     def __init__(self, w: Workload, device: str = "cuda", keep_host: bool = False, n_layers: int = 1,
-                 grouped: bool = True, streaming: bool = False, share_weights: Optional["HotPath"] = None):
+                 grouped: bool = True, streaming: bool = False, share_weights: Optional["HotPath"] = None,
+                 prefetch: bool = True):
         self.grouped = grouped
+        self.prefetch = prefetch
         # decode with the token-by-token scheduler: every step the cached per-sequence state advances by one
         # token (the rows' scores) and the projections take the row gates it emits instead of a chunk table
         self.streaming = streaming
@@ -125,16 +127,37 @@ class HotPath:
             used.update(members)
         return out
 
-    def apply_step(self, table: Optional[cwl.DeviceChunkTable] = None, dense: bool = False, layer: int = 0) -> None:
+    # Decode-sized calls are bound by HBM and spend a large share of the launch draining (partial sums handed over,
+    # outputs stored): each such call is told which weights the NEXT call streams, so that it pulls them towards L2
+    # while it drains.  The order of the calls is static (projection after projection, layer after layer).
+    PREFETCH_MAX_T = 512
+
+    def _next_weights(self, layer: int, i: int, next_layer: Optional[int]) -> Optional[torch.Tensor]:
+        if not self.prefetch or self.T >= self.PREFETCH_MAX_T:
+            return None
+        projs = self.layers[layer]
+        if i + 1 < len(projs):
+            return projs[i + 1].W
+        nl = (layer + 1) % len(self.layers) if next_layer is None else next_layer
+        return self.layers[nl][0].W
+
+    def apply_step(self, table: Optional[cwl.DeviceChunkTable] = None, dense: bool = False, layer: int = 0,
+                   next_layer: Optional[int] = None) -> None:
         if self.streaming and table is None and not dense:
-            for p in self.layers[layer]:
+            for i, p in enumerate(self.layers[layer]):
+                nxt = self._next_weights(layer, i, next_layer)
+                if nxt is not None:
+                    cwl.cwl_prefetch_next(nxt)
                 cwl.cwl_apply_rows(self.X[p.d_in], p.W, p.A, p.B, self.stream_state.gates, Y=p.Y,
                                    workspace=self.apply_ws, status_word=self.status)
             return
         tab = table if table is not None else self.table
-        for group in self.launch_groups(layer):
+        for i, group in enumerate(self.launch_groups(layer)):
             p = group[0]
             if len(group) == 1:
+                nxt = self._next_weights(layer, i, next_layer)
+                if nxt is not None:
+                    cwl.cwl_prefetch_next(nxt)
                 cwl.cwl_apply(self.X[p.d_in], p.W, None if dense else p.A, None if dense else p.B, tab,
                               self.policy.window, Y=p.Y, workspace=self.apply_ws, status_word=self.status)
             else:
@@ -142,11 +165,13 @@ class HotPath:
                                       None if dense else [q.B for q in group], tab, self.policy.window,
                                       Ys=[q.Y for q in group], workspace=self.apply_ws, status_word=self.status)
 
-    def step(self) -> None:
-        """One pass of the whole hot path on the current stream (no host synchronisation)."""
+    def step(self, layer: Optional[int] = None) -> None:
+        """One pass of the whole hot path on the current stream (no host synchronisation): through every layer of
+        the stack, or, with `layer`, through that weight set alone (decode steps rotate over several sets so that
+        no step finds its weights in L2)."""
         if self.streaming:
             self.stream_state.step(self.score)
-        for layer in range(len(self.layers)):
+        for layer in (range(len(self.layers)) if layer is None else (layer,)):
             if self.logits is not None:
                 self.score_step()
             if not self.fixed_table:
@@ -164,7 +189,8 @@ class HotPath:
             self.step()
         return graph
 
-    def launches_per_step(self) -> int:
+    def launches_per_step(self, layers: Optional[int] = None) -> int:
+        """Kernel launches of one step through `layers` weight sets (default: the whole stack)."""
         n = self.LAUNCHES_APPLY * len(self.launch_groups())
         if self.logits is not None:
             n += self.LAUNCHES_SCORE
@@ -172,7 +198,7 @@ class HotPath:
             # up to 32 scan tiles of 2048 scores the tile-sum pass is folded into the prefix pass, and a single
             # sequence has its table written by the walk pass
             n += self.LAUNCHES_PARTITION - (1 if self.T <= 32 * 2048 else 0) - (1 if self.n_seq == 1 else 0)
-        return n * len(self.layers) + (1 if self.streaming else 0)
+        return n * (len(self.layers) if layers is None else layers) + (1 if self.streaming else 0)
 
 
 class HostPipeline:

@@ -38,7 +38,7 @@ def check_projections(w, hp, tab, rows, window):
     for dp, gp in zip(w.projections, hp.projs):
         ref = oracle.apply(w.X[dp.d_in], dp.W, dp.A, dp.B, tab, window, rows=rows)
         got = y_to_f64(gp.Y[torch.from_numpy(rows.astype(np.int64)).cuda()])
-        res = check_output(got, ref, label=f"{w.name} {dp.name} T={w.T}")
+        res = check_output(got, ref, label=f"{w.name} {dp.name} T={w.T}", max_saved_frac=2e-4)
         worst = max(worst, res["rel_fro"])
     return worst
 
