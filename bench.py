@@ -169,7 +169,7 @@ def layers_of(name: str, args) -> int:
     """Weight sets resident on the device: the stack's layers, or the sets a decode run rotates over."""
     if name == "cfg5":
         return args.layers
-    return DECODE_WEIGHT_SETS if name in ("cfg4", "cfg4_stream") else 1
+    return args.weight_sets if name in ("cfg4", "cfg4_stream") else 1
 
 
 def config_dict(name: str, w, n_layers: int, world: int, grouped: bool) -> dict:
@@ -565,7 +565,7 @@ def run_ours(args):
     if args.lean or world > 1:
         cpu = {}
     else:
-        n_rows, _ = rows_for_budget(w, 10.0)         # about 10-20 s of CPU work
+        n_rows, _ = rows_for_budget(w, 25.0)         # about 10-20 s of CPU work
         cpu_val, cpu_info = oracle_sample(w, n_rows=n_rows)
         if stack > 1:
             cpu_val /= stack
@@ -607,6 +607,8 @@ def main():
     ap.add_argument("--layers", type=int, default=32, help="layers of the cfg5 projection stack (a step runs all of them)")
     ap.add_argument("--min-seconds", type=float, default=2.0,
                     help="least device time of a timed region; the block of --steps steps is repeated until it is reached")
+    ap.add_argument("--weight-sets", type=int, default=DECODE_WEIGHT_SETS,
+                    help="distinct weight sets a decode run rotates over (4 x 180 MB > L2, so every step streams from HBM)")
     ap.add_argument("--no-configs", action="store_true", help="headline workload only: no `configs` block")
     ap.add_argument("--no-group", action="store_true",
                     help="one cwl_apply launch per projection instead of grouped launches for q,k,v and gate,up")

@@ -147,6 +147,27 @@ cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64_t ldw,
                      void* workspace, size_t workspace_bytes,
                      int32_t* status_word, void* stream);
 
+/* cwl_apply with a choice of where the cross-fade window lies (Sec. III-D asks for a short window at the join and
+ * does not place it):
+ *   CWL_WINDOW_CAUSAL   the first `window` rows of the incoming chunk (cwl_apply; the only placement a decode step
+ *                       can use, since the incoming configuration is unknown before its chunk opens)
+ *   CWL_WINDOW_CENTRED  the last floor(window/2) rows of the outgoing chunk and the first ceil(window/2) rows of the
+ *                       incoming chunk (prefill: the whole table is known).  Window row i = 0..window-1, counted from
+ *                       the window's first row, has lam = (i+1)/(window+1) for the incoming configuration and
+ *                       1 - lam for the outgoing one.  No window at a join into the first chunk of a sequence.
+ *                       Chunks between two joins should hold at least `window` rows (cwl_partition guarantees it:
+ *                       window <= min_len); where a shorter chunk's two windows meet, the rows go to the join
+ *                       that opened the chunk.
+ * Everything else (arguments, workspace size, shape rules, errors) as cwl_apply; an unknown mode is INVALID_ARG. */
+typedef enum { CWL_WINDOW_CAUSAL = 0, CWL_WINDOW_CENTRED = 1 } cwl_window_mode;
+cwl_status cwl_apply_mode(const void* X, int64_t ldx, const void* W, int64_t ldw,
+                          const void* A, int64_t lda, const void* B, int64_t ldb,
+                          int32_t T, int32_t d_in, int32_t d_out, int32_t R,
+                          cwl_chunk_table table, int32_t window, int32_t window_mode,
+                          void* Y, int64_t ldy,
+                          void* workspace, size_t workspace_bytes,
+                          int32_t* status_word, void* stream);
+
 /* Several adapted projections of the SAME rows in one launch (Sec. III-F: the adapter sits on every attention and
  * MLP projection; q, k, v read one activation, gate and up another).  Projection j computes
  *   Y_j = X W_j + gated (X A_j) B_j

@@ -59,6 +59,7 @@ def lib():
         _lib.cwlo_rung.restype = C.c_int32
         _lib.cwlo_rung.argtypes = [C.c_int64, C.c_int64, C.POINTER(_Policy)]
         _lib.cwlo_blend_weight.restype = C.c_double
+        _lib.cwlo_blend_weight_centred.restype = C.c_double
         _lib.cwlo_get_threads.restype = C.c_int
     return _lib
 
@@ -146,6 +147,35 @@ def partition(score: np.ndarray, cu_seqlens: np.ndarray, ranks, scales, threshol
                       flags[:c].copy(), c)
 
 
+def batch_align(score: np.ndarray, cu_seqlens: np.ndarray, ranks, scales, thresholds, min_len: int, max_len: int,
+                n_buckets: int, window: int = 0, hi_budget: int = -1, capacity: Optional[int] = None):
+    """Batch alignment: sequences bucketed by complexity percentile share their chunk joins.
+    Returns (ChunkTable, bucket [n_seq], order_pos [n_seq])."""
+    s = np.ascontiguousarray(score, dtype=np.float32)
+    cu = np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+    T, n_seq = s.shape[0], cu.shape[0] - 1
+    cap = int(capacity) if capacity is not None else T + n_seq + 1
+    offsets = np.zeros(cap + 1, dtype=np.int32)
+    rank = np.zeros(cap, dtype=np.int32)
+    scale = np.zeros(cap, dtype=np.float32)
+    rung = np.zeros(cap, dtype=np.int32)
+    flags = np.zeros(cap, dtype=np.int32)
+    bucket = np.zeros(max(n_seq, 1), dtype=np.int32)
+    order_pos = np.zeros(max(n_seq, 1), dtype=np.int32)
+    n = C.c_int32(0)
+    p = _policy_struct(ranks, scales, thresholds, min_len, max_len, window, hi_budget)
+    rc = lib().cwlo_batch_align(_ptr(s), _ptr(cu), C.c_int32(n_seq), C.c_int32(T), C.byref(p), C.c_int32(n_buckets),
+                                _ptr(offsets), _ptr(rank), _ptr(scale), _ptr(rung), _ptr(flags),
+                                C.byref(n), C.c_int32(cap), _ptr(bucket), _ptr(order_pos))
+    if rc == 4:
+        raise OverflowError("cwlo_batch_align: chunk table capacity exceeded")
+    if rc != 0:
+        raise ValueError(f"cwlo_batch_align: status {rc}")
+    c = n.value
+    tab = ChunkTable(offsets[:c + 1].copy(), rank[:c].copy(), scale[:c].copy(), rung[:c].copy(), flags[:c].copy(), c)
+    return tab, bucket[:n_seq].copy(), order_pos[:n_seq].copy()
+
+
 def blend_weights(table: ChunkTable, T: int, window: int) -> np.ndarray:
     """Weight of the incoming configuration for every row (fp64 [T])."""
     off = np.ascontiguousarray(table.offsets, dtype=np.int32)
@@ -157,9 +187,26 @@ def blend_weights(table: ChunkTable, T: int, window: int) -> np.ndarray:
     return out
 
 
+def blend_weights_centred(table: ChunkTable, T: int, window: int):
+    """Centred window placement: (weight of cfg_in, cfg_in, cfg_out) for every row."""
+    off = np.ascontiguousarray(table.offsets, dtype=np.int32)
+    fl = np.ascontiguousarray(table.flags, dtype=np.int32)
+    lam = np.empty(T, dtype=np.float64)
+    cin = np.empty(T, dtype=np.int32)
+    cout = np.empty(T, dtype=np.int32)
+    f = lib().cwlo_blend_weight_centred
+    a, b = C.c_int32(0), C.c_int32(0)
+    for t in range(T):
+        lam[t] = f(C.c_int32(t), _ptr(off), _ptr(fl), C.c_int32(table.n_chunks), C.c_int32(window), C.byref(a), C.byref(b))
+        cin[t], cout[t] = a.value, b.value
+    return lam, cin, cout
+
+
 def apply(X: np.ndarray, W: np.ndarray, A: Optional[np.ndarray], B: Optional[np.ndarray],
-          table: Optional[ChunkTable], window: int, rows: Optional[np.ndarray] = None) -> np.ndarray:
+          table: Optional[ChunkTable], window: int, rows: Optional[np.ndarray] = None,
+          centred: bool = False) -> np.ndarray:
     """Adapted projection in fp64.  X, W, A, B are uint16 arrays of bf16 bit patterns.
+    ``centred`` places the cross-fade window around each join instead of after it.
 
     Returns Y [T, d_out] or, with ``rows``, Y [len(rows), d_out] in list order."""
     X = np.ascontiguousarray(X, dtype=np.uint16)
@@ -190,7 +237,8 @@ def apply(X: np.ndarray, W: np.ndarray, A: Optional[np.ndarray], B: Optional[np.
     else:
         off = rk = sc = fl = None
         nc = 0
-    rc = lib().cwlo_apply(_ptr(X), C.c_int64(d_in), _ptr(W), C.c_int64(d_out),
+    fn = lib().cwlo_apply_centred if centred else lib().cwlo_apply
+    rc = fn(_ptr(X), C.c_int64(d_in), _ptr(W), C.c_int64(d_out),
                           _ptr(A), C.c_int64(R), _ptr(B), C.c_int64(d_out),
                           C.c_int32(T), C.c_int32(d_in), C.c_int32(d_out), C.c_int32(R),
                           _ptr(off), _ptr(rk), _ptr(sc), _ptr(fl), C.c_int32(nc), C.c_int32(window),

@@ -278,6 +278,242 @@ int cwlo_apply(const uint16_t* X, int64_t ldx, const uint16_t* W, int64_t ldw,
 }
 
 /* ---------------------------------------------------------------------------------------------
+ * Sec. III-G / IV-F, batch alignment: sequences of a batch are bucketed by complexity percentile so that the
+ * chunk joins of a bucket line up, while every sequence keeps its own rank choices.  The paper gives one
+ * sentence; this build's reading, step by step:
+ *   1. the complexity of a sequence is the mean of its quantised scores (sum_n / len_n, compared exactly by
+ *      cross-multiplication); sequences are ordered by it, ascending, the lower index first on ties, empty
+ *      sequences before all others;
+ *   2. the sequence at position i of that order (0-based) falls into bucket floor(i * n_buckets / n_seq):
+ *      percentile bands of (almost) equal population;
+ *   3. per bucket the scores are pooled position by position (positions count from each sequence's start):
+ *      S[j] = sum of q over the members that have a token at position j, N[j] = how many do;
+ *   4. the greedy walk of Sec. III-B (cwlo_partition's rule) runs ONCE per bucket on the pooled track over
+ *      positions [0, longest member): the mean of a span is sum S / sum N, i.e. the mean over all member
+ *      tokens at those positions; its cuts are the bucket's shared joins;
+ *   5. a member takes every shared join that leaves it at least L_min tokens (join <= len_n - L_min), so
+ *      its last chunk absorbs what a later join would have cut off too short;
+ *   6. rung, budget, rank and scale of each chunk come from the sequence's OWN scores, as in cwlo_partition.
+ * Outputs: the chunk table in sequence order, bucket[n] and order_pos[n] (position of sequence n in the
+ * complexity order).
+ * ------------------------------------------------------------------------------------------- */
+static int32_t pooled_rung(int64_t sum, int64_t count, const cwlo_policy* p) {
+  int32_t k = 0;
+  for (int32_t j = 0; j + 1 < p->n_rungs; ++j)
+    if (sum >= threshold_q(p->threshold[j]) * count) ++k;
+  return k;
+}
+
+int cwlo_batch_align(const float* score, const int32_t* cu, int32_t n_seq, int32_t T,
+                     const cwlo_policy* p, int32_t n_buckets,
+                     int32_t* offsets, int32_t* rank, float* scale, int32_t* rung, int32_t* flags,
+                     int32_t* n_chunks, int32_t capacity, int32_t* bucket, int32_t* order_pos) {
+  if (!score || !cu || !offsets || !rank || !scale || !rung || !flags || !n_chunks || !bucket || !order_pos)
+    return CWLO_ERR_ARG;
+  if (n_seq < 0 || T < 0 || capacity < 0 || n_buckets < 1 || !policy_ok(p)) return CWLO_ERR_ARG;
+  if (cu[0] != 0 || cu[n_seq] != T) return CWLO_ERR_ARG;
+  for (int32_t n = 0; n < n_seq; ++n)
+    if (cu[n + 1] < cu[n]) return CWLO_ERR_ARG;
+  const int32_t Lmin = p->min_len, Lmax = p->max_len, K = p->n_rungs;
+
+  int64_t* P = (int64_t*)malloc(sizeof(int64_t) * ((size_t)T + 1));      /* prefix sums of the packed scores */
+  int64_t* PS = (int64_t*)malloc(sizeof(int64_t) * ((size_t)T + 2));     /* pooled track of one bucket, prefix sums */
+  int64_t* PN = (int64_t*)malloc(sizeof(int64_t) * ((size_t)T + 2));
+  int32_t* joins = (int32_t*)malloc(sizeof(int32_t) * ((size_t)T + 2));
+  P[0] = 0;
+  for (int32_t t = 0; t < T; ++t) P[t + 1] = P[t] + cwlo_quantise(score[t]);
+
+  /* 1./2. complexity order and percentile buckets */
+  for (int32_t n = 0; n < n_seq; ++n) {
+    const int64_t sum_n = P[cu[n + 1]] - P[cu[n]], len_n = cu[n + 1] - cu[n];
+    int32_t before = 0;
+    for (int32_t m = 0; m < n_seq; ++m) {
+      if (m == n) continue;
+      const int64_t sum_m = P[cu[m + 1]] - P[cu[m]], len_m = cu[m + 1] - cu[m];
+      int m_first;
+      if (len_m == 0 || len_n == 0) {
+        if (len_m == 0 && len_n == 0) m_first = m < n;
+        else m_first = (len_m == 0);
+      } else {
+        const int64_t lhs = sum_m * len_n, rhs = sum_n * len_m;          /* mean_m against mean_n */
+        m_first = lhs < rhs || (lhs == rhs && m < n);
+      }
+      if (m_first) ++before;
+    }
+    order_pos[n] = before;
+    bucket[n] = (int32_t)(((int64_t)before * n_buckets) / n_seq);
+  }
+
+  int32_t C = 0;
+  int status = CWLO_OK;
+  offsets[0] = 0;
+  /* chunks are emitted in sequence order; the shared joins of a sequence's bucket are worked out when needed */
+  for (int32_t n = 0; n < n_seq && status == CWLO_OK; ++n) {
+    const int32_t S = cu[n], len_n = cu[n + 1] - cu[n], k = bucket[n];
+    if (len_n == 0) continue;
+    /* 3. pooled track of bucket k */
+    int32_t L = 0;
+    for (int32_t m = 0; m < n_seq; ++m)
+      if (bucket[m] == k && cu[m + 1] - cu[m] > L) L = cu[m + 1] - cu[m];
+    PS[0] = 0; PN[0] = 0;
+    for (int32_t j = 0; j < L; ++j) {
+      int64_t s = 0, c = 0;
+      for (int32_t m = 0; m < n_seq; ++m)
+        if (bucket[m] == k && cu[m + 1] - cu[m] > j) { s += cwlo_quantise(score[cu[m] + j]); c += 1; }
+      PS[j + 1] = PS[j] + s; PN[j + 1] = PN[j] + c;
+    }
+    /* 4. the walk of Sec. III-B on the pooled track over [0, L) */
+    int32_t n_joins = 0;
+    int32_t b = 0;
+    while (b < L) {
+      int32_t e;
+      if (L - b < 2 * Lmin) {
+        e = L;
+      } else {
+        e = b + Lmin;
+        for (;;) {
+          if (e - b >= Lmax) break;
+          int32_t open_rung  = pooled_rung(PS[e] - PS[b], PN[e] - PN[b], p);
+          int32_t ahead_rung = pooled_rung(PS[e + Lmin] - PS[e], PN[e + Lmin] - PN[e], p);
+          if (open_rung != ahead_rung) break;
+          e = e + 1;
+          if (L - e < Lmin) { e = L; break; }
+        }
+      }
+      if (e < L) joins[n_joins++] = e;
+      b = e;
+    }
+    /* 5. the member's own chunks */
+    const int32_t first_chunk = C;
+    int32_t start = 0;
+    for (int32_t i = 0; i <= n_joins && status == CWLO_OK; ++i) {
+      int32_t end;
+      if (i < n_joins && joins[i] <= len_n - Lmin) end = joins[i];
+      else end = len_n;
+      if (C >= capacity) { status = CWLO_ERR_CAPACITY; break; }
+      offsets[C + 1] = S + end;
+      flags[C] = (start == 0) ? 1 : 0;
+      rung[C] = cwlo_rung(P[S + end] - P[S + start], end - start, p);     /* 6. own scores */
+      ++C;
+      start = end;
+      if (end == len_n) break;
+    }
+    if (status != CWLO_OK) break;
+    /* 6. budget on top-rung chunks, per sequence, exactly as in cwlo_partition */
+    if (p->hi_budget >= 0 && K >= 2 && C > first_chunk) {
+      int32_t* walked = (int32_t*)malloc(sizeof(int32_t) * (size_t)(C - first_chunk));
+      for (int32_t c = first_chunk; c < C; ++c) walked[c - first_chunk] = rung[c];
+      for (int32_t c = first_chunk; c < C; ++c) {
+        if (walked[c - first_chunk] != K - 1) continue;
+        int64_t sum_c = P[offsets[c + 1]] - P[offsets[c]], len_c = offsets[c + 1] - offsets[c];
+        int32_t better = 0;
+        for (int32_t d = first_chunk; d < C; ++d) {
+          if (d == c || walked[d - first_chunk] != K - 1) continue;
+          int64_t sum_d = P[offsets[d + 1]] - P[offsets[d]], len_d = offsets[d + 1] - offsets[d];
+          int64_t lhs = sum_d * len_c, rhs = sum_c * len_d;
+          if (lhs > rhs || (lhs == rhs && d < c)) ++better;
+        }
+        if (better >= p->hi_budget) rung[c] = K - 2;
+      }
+      free(walked);
+    }
+  }
+  if (status == CWLO_OK) {
+    for (int32_t c = 0; c < C; ++c) {
+      rank[c] = p->rung_rank[rung[c]];
+      scale[c] = p->rung_scale[rung[c]];
+    }
+    *n_chunks = C;
+  }
+  free(P); free(PS); free(PN); free(joins);
+  return status;
+}
+
+/* ---------------------------------------------------------------------------------------------
+ * Sec. III-D, centred placement of the cross-fade window (a variant: the paper says only that the
+ * window is short).  The w rows AROUND a join are blended: the last floor(w/2) rows of the outgoing
+ * chunk and the first ceil(w/2) rows of the incoming chunk.  Counted from the window's first row,
+ * row i = 0..w-1 gets the weight (i+1)/(w+1) for the incoming configuration, as in the causal
+ * placement.  A join into the first chunk of a sequence has no window.  Where a chunk is so short
+ * that the window after its opening join and the one before its closing join meet, the rows of the
+ * opening join's window win.
+ *   returns lam, the weight of configuration *cfg_in; *cfg_out carries 1 - lam (equal to *cfg_in
+ *   and lam = 1 outside every window).
+ * ------------------------------------------------------------------------------------------- */
+double cwlo_blend_weight_centred(int32_t t, const int32_t* offsets, const int32_t* flags,
+                                 int32_t n_chunks, int32_t window, int32_t* cfg_in, int32_t* cfg_out) {
+  int32_t c = 0;
+  while (c + 1 < n_chunks && offsets[c + 1] <= t) ++c;
+  const int32_t before = window / 2;          /* rows of the window in the outgoing chunk */
+  const int32_t after = window - before;      /* rows of the window in the incoming chunk */
+  const int32_t j = t - offsets[c];
+  const int32_t len = offsets[c + 1] - offsets[c];
+  int32_t in = c, out = c;
+  double lam = 1.0;
+  if (c > 0 && !(flags[c] & 1) && j < after) {
+    /* head of the incoming chunk: window row i = before + j */
+    lam = (double)(before + j + 1) / (double)(window + 1);
+    in = c; out = c - 1;
+  } else if (c + 1 < n_chunks && !(flags[c + 1] & 1) && len - j <= before) {
+    /* tail of the outgoing chunk: the window starts `before` rows ahead of the join */
+    lam = (double)(before - (len - j) + 1) / (double)(window + 1);
+    in = c + 1; out = c;
+  }
+  if (cfg_in) *cfg_in = in;
+  if (cfg_out) *cfg_out = out;
+  return lam;
+}
+
+/* Adapted projection with the centred window: for a row whose window joins configurations `out` and `in`,
+ *   y_t = x_t W + (1-lam_t) s_out (x_t A[:, :r_out]) B[:r_out, :] + lam_t s_in (x_t A[:, :r_in]) B[:r_in, :],
+ * the three products computed one by one and then combined.  Arguments as cwlo_apply. */
+int cwlo_apply_centred(const uint16_t* X, int64_t ldx, const uint16_t* W, int64_t ldw,
+                       const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
+                       int32_t T, int32_t d_in, int32_t d_out, int32_t R,
+                       const int32_t* offsets, const int32_t* rank, const float* scale,
+                       const int32_t* flags, int32_t n_chunks, int32_t window,
+                       const int32_t* rows, int32_t n_rows, double* Y, int64_t ldy) {
+  if (!X || !W || !Y || T < 0 || d_in < 1 || d_out < 1 || R < 0 || window < 0) return CWLO_ERR_ARG;
+  const int has_adapter = (A != NULL && B != NULL && R > 0);
+  if (has_adapter) {
+    if (!offsets || !rank || !scale || !flags || n_chunks < 1) return CWLO_ERR_ARG;
+    if (offsets[0] != 0 || offsets[n_chunks] != T) return CWLO_ERR_ARG;
+    for (int32_t c = 0; c < n_chunks; ++c)
+      if (rank[c] < 0 || rank[c] > R || offsets[c + 1] < offsets[c]) return CWLO_ERR_ARG;
+  }
+  const int32_t count = rows ? n_rows : T;
+  int bad = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int32_t i = 0; i < count; ++i) {
+    const int32_t t = rows ? rows[i] : i;
+    if (t < 0 || t >= T) { bad = 1; continue; }
+    const uint16_t* x = X + (int64_t)t * ldx;
+    double* y = Y + (int64_t)i * ldy;
+    for (int32_t n = 0; n < d_out; ++n) y[n] = 0.0;
+    for (int32_t k = 0; k < d_in; ++k) {
+      double xk = bf16_to_double(x[k]);
+      const uint16_t* w = W + (int64_t)k * ldw;
+      for (int32_t n = 0; n < d_out; ++n) y[n] += xk * bf16_to_double(w[n]);
+    }
+    if (!has_adapter) continue;
+    int32_t in, out;
+    double lam = cwlo_blend_weight_centred(t, offsets, flags, n_chunks, window, &in, &out);
+    double* h = (double*)malloc(sizeof(double) * (size_t)(R > 0 ? R : 1));
+    double* d_new = (double*)malloc(sizeof(double) * (size_t)d_out);
+    double* d_old = (double*)malloc(sizeof(double) * (size_t)d_out);
+    adapter_row(x, A, lda, B, ldb, d_in, d_out, rank[in], (double)scale[in], h, d_new);
+    if (lam < 1.0) {
+      adapter_row(x, A, lda, B, ldb, d_in, d_out, rank[out], (double)scale[out], h, d_old);
+      for (int32_t n = 0; n < d_out; ++n) y[n] += (1.0 - lam) * d_old[n] + lam * d_new[n];
+    } else {
+      for (int32_t n = 0; n < d_out; ++n) y[n] += d_new[n];
+    }
+    free(h); free(d_new); free(d_old);
+  }
+  return bad ? CWLO_ERR_ARG : CWLO_OK;
+}
+
+/* ---------------------------------------------------------------------------------------------
  * Decode-time scheduler (Sec. III-A, III-B, III-F: scores arrive as tokens stream in, tokens are
  * grouped as they arrive, and the scheduler keeps its state from step to step).  The paper names the constraints only; the rule is
  * this build's causal reading: a token may open a new chunk only on what has been seen so far.

@@ -20,6 +20,10 @@
  *   budget    pinned  (definition: keep the H largest means, earlier index wins ties)
  *   blend     pinned  (weights sum to one, equal spacing, convex combination of single-chunk runs)
  *   apply     pinned  (merged-weight LoRA, r = 0 base, hand-expanded tiny case, linearity)
+ *   align     parity unpinned against the paper (one sentence, no rule); pinned internally: one bucket per sequence
+ *             reduces to the pinned cwlo_partition, a hand-traced pooled walk, invariants, an exact-rational brute force
+ *   centred   pinned  (window sums, equal spacing, the causal ramp shifted, convex combination of single-
+ *             configuration runs, hand-expanded tiny case)
  *   mixed     pinned  (weights (1,0,0) = entropy score, hand-traced novelty, closed-form prior, set-based brute force)
  *   stream    parity unpinned against the paper (no rule printed); pinned internally by hand-traced runs,
  *             invariants and an independent brute force; apply_rows pinned against cwlo_apply on equivalent tables
@@ -91,6 +95,28 @@ int cwlo_apply(const uint16_t* X, int64_t ldx, const uint16_t* W, int64_t ldw,
                const int32_t* offsets, const int32_t* rank, const float* scale,
                const int32_t* flags, int32_t n_chunks, int32_t window,
                const int32_t* rows, int32_t n_rows, double* Y, int64_t ldy);
+
+/* Batch alignment (Sec. III-G, IV-F): sequences are bucketed by complexity percentile and the members of a
+ * bucket share their chunk joins (worked out on the bucket's pooled score track), while rung, budget, rank
+ * and scale stay per sequence.  See cwlo.c for the steps.  Table outputs as cwlo_partition;
+ * bucket[n_seq] and order_pos[n_seq] receive each sequence's bucket and its position in the complexity order. */
+int cwlo_batch_align(const float* score, const int32_t* cu_seqlens, int32_t n_seq, int32_t T,
+                     const cwlo_policy* p, int32_t n_buckets,
+                     int32_t* offsets, int32_t* rank, float* scale, int32_t* rung, int32_t* flags,
+                     int32_t* n_chunks, int32_t capacity, int32_t* bucket, int32_t* order_pos);
+
+/* The cross-fade window placed AROUND the join instead of after it (Sec. III-D variant): the last
+ * floor(w/2) rows of the outgoing chunk and the first ceil(w/2) rows of the incoming chunk; window
+ * row i gets (i+1)/(w+1) for the incoming configuration.  Returns that weight; *cfg_in / *cfg_out
+ * receive the chunk indices whose (rank, scale) carry lam and 1 - lam. */
+double cwlo_blend_weight_centred(int32_t t, const int32_t* offsets, const int32_t* flags,
+                                 int32_t n_chunks, int32_t window, int32_t* cfg_in, int32_t* cfg_out);
+int cwlo_apply_centred(const uint16_t* X, int64_t ldx, const uint16_t* W, int64_t ldw,
+                       const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
+                       int32_t T, int32_t d_in, int32_t d_out, int32_t R,
+                       const int32_t* offsets, const int32_t* rank, const float* scale,
+                       const int32_t* flags, int32_t n_chunks, int32_t window,
+                       const int32_t* rows, int32_t n_rows, double* Y, int64_t ldy);
 
 /* Mix of complexity signals (Sec. III-A (i), (ii), (iv)); see cwlo.c for the definitions. */
 typedef struct {

@@ -23,8 +23,9 @@ EXPORTS = ["cwl_status_string", "cwl_version", "cwl_score_tokens", "cwl_score_to
            "cwl_partition", "cwl_apply_workspace_bytes", "cwl_apply", "cwl_apply_grouped_workspace_bytes",
            "cwl_apply_grouped", "cwl_apply_plan", "cwl_stream_state_bytes", "cwl_stream_reset", "cwl_stream_step",
            "cwl_apply_rows", "cwl_ladder_workspace_bytes", "cwl_ladder_build", "cwl_debug_set",
-           "cwl_apply_noalloc_scratch_need", "cwl_apply_noalloc", "cwl_prefetch_next"]
+           "cwl_apply_noalloc_scratch_need", "cwl_apply_noalloc", "cwl_prefetch_next", "cwl_apply_mode"]
 NOALLOC_SCRATCH_BYTES = 8 << 20
+WINDOW_CAUSAL, WINDOW_CENTRED = 0, 1
 
 
 class CwlError(RuntimeError):
@@ -108,6 +109,10 @@ def lib():
                                 C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                 CChunkTable, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t,
                                 C.c_void_p, C.c_void_p]
+        L.cwl_apply_mode.restype = C.c_int
+        L.cwl_apply_mode.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
+                                     C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32, CChunkTable,
+                                     C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         L.cwl_apply_grouped_workspace_bytes.restype = C.c_size_t
         L.cwl_apply_grouped_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_int32), C.c_int32]
         L.cwl_apply_grouped.restype = C.c_int
@@ -282,8 +287,9 @@ def cwl_apply_noalloc_scratch_need(T: int, d_in: int, d_out: int, R: int) -> int
 def cwl_apply(X: torch.Tensor, W: torch.Tensor, A: Optional[torch.Tensor], B: Optional[torch.Tensor],
               table: Optional[DeviceChunkTable], window: int, Y: Optional[torch.Tensor] = None,
               workspace: Optional[torch.Tensor] = None, status_word: Optional[torch.Tensor] = None,
-              stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
-    """Y = X W + gated (X A) B per the chunk table (bf16 tensors on the device, row-major)."""
+              stream: Optional[torch.cuda.Stream] = None, centred: bool = False) -> torch.Tensor:
+    """Y = X W + gated (X A) B per the chunk table (bf16 tensors on the device, row-major).  ``centred`` places the
+    cross-fade window around each join (cwl_apply_mode) instead of after it."""
     for t in (X, W):
         assert t.is_cuda and t.dtype == torch.bfloat16 and t.dim() == 2 and t.stride(1) == 1
     T, d_in = X.shape
@@ -298,6 +304,12 @@ def cwl_apply(X: torch.Tensor, W: torch.Tensor, A: Optional[torch.Tensor], B: Op
     if workspace is None:
         workspace = torch.empty(need, dtype=torch.uint8, device=X.device)
     ct = table.c_struct() if table is not None else CChunkTable(None, None, None, None, None, None, 0)
+    if centred:
+        _check("cwl_apply_mode", lib().cwl_apply_mode(_p(X), X.stride(0), _p(W), W.stride(0),
+                                                      _p(A), A.stride(0) if R else 0, _p(B), B.stride(0) if R else 0,
+                                                      T, d_in, d_out, R, ct, int(window), WINDOW_CENTRED, _p(Y), Y.stride(0),
+                                                      _p(workspace), workspace.numel(), _p(status_word), _stream_ptr(stream)))
+        return Y
     _check("cwl_apply", lib().cwl_apply(_p(X), X.stride(0), _p(W), W.stride(0),
                                         _p(A), A.stride(0) if R else 0, _p(B), B.stride(0) if R else 0,
                                         T, d_in, d_out, R, ct, int(window), _p(Y), Y.stride(0),

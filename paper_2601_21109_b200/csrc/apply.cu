@@ -97,6 +97,7 @@ struct ApplyParams {
   int T, d_in, R;          // R = 0: no adapter
   int RT;                  // n_proj * R: columns of the shrink output, all projections side by side
   int window;
+  int window_mode;         // CWL_WINDOW_CAUSAL: the window follows the join; CWL_WINDOW_CENTRED: it lies around it
   __nv_bfloat16* Y[CWL_MAX_GROUP]; int64_t ldy[CWL_MAX_GROUP];
   __nv_bfloat16* Hg;       // [T, RT] gated shrink outputs
   float* partial;          // [shrink_splits, 128-row tiles, RT / 4, 128, 4] fp32 partial shrink sums
@@ -397,12 +398,28 @@ __device__ __forceinline__ RowGate row_gate(int t, const ApplyParams& p) {
     }
     const int c = lo, j = t - tb.offsets[c];
     float lam = 1.f;
-    if (c > 0 && !(tb.flags[c] & 1) && j < p.window) lam = (float)(j + 1) / (float)(p.window + 1);
-    g.r_in = min(max(tb.rank[c], 0), p.R);
-    g.w_in = lam * tb.scale[c];
+    int c_in = c, c_out = c;                       // configurations carrying lam and 1 - lam
+    if (p.window_mode == CWL_WINDOW_CENTRED) {
+      // the window lies around the join: floor(w/2) rows before it, ceil(w/2) rows after it; where a short chunk's
+      // two windows meet, the rows belong to the join that opened the chunk
+      const int before = p.window >> 1, after = p.window - before;
+      const int len = tb.offsets[c + 1] - tb.offsets[c];
+      if (c > 0 && !(tb.flags[c] & 1) && j < after) {
+        lam = (float)(before + j + 1) / (float)(p.window + 1);
+        c_out = c - 1;
+      } else if (c + 1 < C && !(tb.flags[c + 1] & 1) && len - j <= before) {
+        lam = (float)(before - (len - j) + 1) / (float)(p.window + 1);
+        c_in = c + 1;
+      }
+    } else if (c > 0 && !(tb.flags[c] & 1) && j < p.window) {
+      lam = (float)(j + 1) / (float)(p.window + 1);
+      c_out = c - 1;
+    }
+    g.r_in = min(max(tb.rank[c_in], 0), p.R);
+    g.w_in = lam * tb.scale[c_in];
     if (lam < 1.f) {
-      g.r_out = min(max(tb.rank[c - 1], 0), p.R);
-      g.w_out = (1.f - lam) * tb.scale[c - 1];
+      g.r_out = min(max(tb.rank[c_out], 0), p.R);
+      g.w_out = (1.f - lam) * tb.scale[c_out];
     }
   }
   return g;
@@ -1305,7 +1322,8 @@ cwl_status check_group(const void* X, int64_t ldx, const cwl_projection* proj, i
 cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* proj, int n_proj, int32_t T,
                             int32_t d_in, int32_t R, cwl_chunk_table table, int32_t window, void* workspace,
                             size_t workspace_bytes, int32_t* status_word, void* stream_, bool allow_split_k,
-                            size_t scratch_limit, const cwl_row_gate* row_gates = nullptr) {
+                            size_t scratch_limit, const cwl_row_gate* row_gates = nullptr,
+                            int32_t window_mode = CWL_WINDOW_CAUSAL) {
   // the calling thread's one-shot prefetch hint belongs to this call, whatever becomes of it
   const NextPrefetch hint = t_next_prefetch;
   t_next_prefetch = {nullptr, 0};
@@ -1346,7 +1364,7 @@ cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* pr
 
   ApplyParams p{};
   p.T = T; p.d_in = d_in; p.R = Reff; p.RT = n_proj * Reff;
-  p.window = window;
+  p.window = window; p.window_mode = window_mode;
   for (int j = 0; j < n_proj; ++j) { p.Y[j] = static_cast<__nv_bfloat16*>(proj[j].Y); p.ldy[j] = proj[j].ldy; }
   p.Hg = ws.Hg; p.partial = ws.partial; p.sk_partial = ws.sk_partial;
   p.counters = ws.sync; p.flags = ws.sync + 2 * pl.n_m_pairs * n_proj; p.sk_counters = ws.sync + 4 * pl.n_m_pairs * n_proj;
@@ -1397,13 +1415,13 @@ cwl_status apply_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, co
                       const void* B, int64_t ldb, int32_t T, int32_t d_in, int32_t d_out, int32_t R,
                       cwl_chunk_table table, int32_t window, void* Y, int64_t ldy, void* workspace,
                       size_t workspace_bytes, int32_t* status_word, void* stream, bool allow_split_k,
-                      size_t scratch_limit = 0) {
+                      size_t scratch_limit = 0, int32_t window_mode = CWL_WINDOW_CAUSAL) {
   const bool adapter = (A != nullptr && B != nullptr && R > 0);
   cwl_projection q;
   q.W = W; q.ldw = ldw; q.A = adapter ? A : nullptr; q.lda = lda; q.B = adapter ? B : nullptr; q.ldb = ldb;
   q.Y = Y; q.ldy = ldy; q.d_out = d_out;
   return apply_group_impl(X, ldx, &q, 1, T, d_in, R, table, window, workspace, workspace_bytes, status_word, stream,
-                          allow_split_k, scratch_limit);
+                          allow_split_k, scratch_limit, nullptr, window_mode);
 }
 
 }  // namespace
@@ -1457,6 +1475,17 @@ extern "C" cwl_status cwl_apply(const void* X, int64_t ldx, const void* W, int64
                                 int32_t* status_word, void* stream) {
   return cwl::apply_impl(X, ldx, W, ldw, A, lda, B, ldb, T, d_in, d_out, R, table, window, Y, ldy, workspace,
                          workspace_bytes, status_word, stream, true);
+}
+
+extern "C" cwl_status cwl_apply_mode(const void* X, int64_t ldx, const void* W, int64_t ldw,
+                                     const void* A, int64_t lda, const void* B, int64_t ldb,
+                                     int32_t T, int32_t d_in, int32_t d_out, int32_t R,
+                                     cwl_chunk_table table, int32_t window, int32_t window_mode,
+                                     void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
+                                     int32_t* status_word, void* stream) {
+  if (window_mode != CWL_WINDOW_CAUSAL && window_mode != CWL_WINDOW_CENTRED) return CWL_ERR_INVALID_ARG;
+  return cwl::apply_impl(X, ldx, W, ldw, A, lda, B, ldb, T, d_in, d_out, R, table, window, Y, ldy, workspace,
+                         workspace_bytes, status_word, stream, true, 0, window_mode);
 }
 
 extern "C" size_t cwl_apply_grouped_workspace_bytes(int32_t T, int32_t d_in, int32_t n_proj, const int32_t* d_out,
