@@ -124,6 +124,33 @@ cwl_status cwl_partition(const float* score, const int32_t* cu_seqlens, int32_t 
                          void* workspace, size_t workspace_bytes,
                          int32_t* status_word, void* stream);
 
+/* Batch alignment (Sec. III-G: sequences of a batch are bucketed by complexity percentile so that chunk joins line
+ * up across the batch, while each sequence still makes its own rank choices; Sec. IV-F names a batch alignment
+ * controller).  The paper gives no rule; the one used here, an alternative to cwl_partition for a packed batch:
+ *   1. a sequence's complexity is the mean of its quantised scores (exact integer compares); sequences are ordered
+ *      by it, ascending, lower index first on ties, empty sequences first: order_pos[n] is n's position;
+ *   2. bucket[n] = floor(order_pos[n] * n_buckets / n_seq): percentile bands of near-equal population;
+ *   3. per bucket the scores are pooled position by position, counted from each member's start (sum of the
+ *      members' quantised scores at position j, and how many members reach j);
+ *   4. cwl_partition's greedy walk runs once per bucket on the pooled track, over the positions of its longest
+ *      member; the mean of a span is the mean over all member tokens at those positions.  Its cuts are the
+ *      bucket's shared joins;
+ *   5. a member takes every shared join that leaves it at least min_len tokens; its last chunk absorbs the rest
+ *      (so a chunk is shorter than max_len + min_len, as with cwl_partition);
+ *   6. rung, hi_budget, rank and scale of a chunk come from the sequence's own scores, as in cwl_partition.
+ * With n_buckets >= n_seq every sequence is alone in its bucket and the table equals cwl_partition's.
+ *   score, cu_seqlens, policy, table, status_word   as for cwl_partition (same capacity rule and CAPACITY flag)
+ *   bucket, order_pos   DEV int32 [n_seq], outputs
+ *   workspace           DEV, cwl_batch_align_workspace_bytes(T, n_seq, n_buckets) bytes, 16-byte aligned
+ * Errors: INVALID_ARG (NULLs, bad policy, n_buckets < 1), UNSUPPORTED (T > 2^19 tokens or n_buckets > 1024),
+ * WORKSPACE, CUDA.  Scheduler-level work: nine small launches, no host synchronisation. */
+size_t     cwl_batch_align_workspace_bytes(int32_t T, int32_t n_seq, int32_t n_buckets);
+cwl_status cwl_batch_align(const float* score, const int32_t* cu_seqlens, int32_t n_seq, int32_t T,
+                           const cwl_policy* policy, int32_t n_buckets, cwl_chunk_table table,
+                           int32_t* bucket, int32_t* order_pos,
+                           void* workspace, size_t workspace_bytes,
+                           int32_t* status_word, void* stream);
+
 /* Adapted projection (Sec. III-F) with the boundary-safe cross-fade (Sec. III-D):
  *   y_t = x_t W + (1 - lam_t) s_p (x_t A[:, :r_p]) B[:r_p, :] + lam_t s_c (x_t A[:, :r_c]) B[:r_c, :]
  * for row t in chunk c with predecessor p = c - 1.  Rows j = 0..window-1 of a chunk that is not
@@ -250,6 +277,18 @@ cwl_status cwl_ladder_build(const void* A, int64_t lda, const void* B, int64_t l
                             float* A_out_f32, float* B_out_f32, float* sigma,
                             void* workspace, size_t workspace_bytes, int32_t* sweeps, void* stream);
 
+/* How much of the GPU the apply calls of THIS host thread plan for: at most `pairs` CTA pairs (2 SMs each; a B200
+ * holds 74), 0 = all of them (the default).  Independent projections -- no one reads what another writes -- can then
+ * run side by side on different streams, each on its share of the SMs, so that one call's set-up and drain (partial
+ * sums handed over, outputs stored) overlap the other's weight stream; it matters for decode-sized calls, whose
+ * set-up and drain are a large share of the launch (Sec. III-F puts the adapter on every attention and MLP
+ * projection, and the projections of one step that read ready inputs are independent).  The budget also enters
+ * cwl_apply_workspace_bytes and cwl_apply_plan-style decisions made by later calls of the thread; calls that run
+ * side by side need distinct workspaces.  Budgets of concurrent calls should add up to the resident pairs or less:
+ * a call's waits only make progress once all its pairs are resident (they are bounded, see CWL_ERR_TIMEOUT).
+ * Errors: INVALID_ARG (pairs < 0). */
+cwl_status cwl_set_pair_budget(int32_t pairs);
+
 /* One-shot hint for the NEXT cwl_apply / cwl_apply_rows / cwl_apply_grouped call made by this host thread: the
  * region [ptr, ptr + bytes) is what the call AFTER that one will stream -- typically the weight matrix of the
  * projection that follows (weights and adapter factors are frozen at inference: Sec. III-C).  Once a CTA of the
@@ -262,13 +301,6 @@ cwl_status cwl_ladder_build(const void* A, int64_t lda, const void* B, int64_t l
  * The hint is consumed by the next call whether or not that call launches anything; it has no effect on results.
  * Thread-local; no device work is done by this call itself. */
 cwl_status cwl_prefetch_next(const void* ptr, size_t bytes);
-
-/* Test hook for the failure path of cwl_apply and its variants.  Every device-side wait (mbarrier, H' flag, split-K
- * counter) is bounded; when one runs out the CTA raises CWL_ERR_TIMEOUT in *status_word (bit 1 << CWL_ERR_TIMEOUT),
- * drains its copies, frees its tensor memory and returns, so the context stays usable.  This call sets the limit
- * (ns; <= 0 restores the default of 2 s) and, with withhold_publish != 0, makes the shrink never publish H', so that
- * the waits on it run out.  Process-wide, not thread-safe, not for production use. */
-void cwl_debug_set(int64_t wait_limit_ns, int32_t withhold_publish);
 
 /* The schedule cwl_apply uses for a shape when `pairs` CTA pairs can be resident (a B200 holds 74): how
  * the output is cut into column tiles (Sec. III-F leaves the kernel schedule open; this is the library's own

@@ -1,0 +1,31 @@
+/*
+ * cwl_test_hooks.h -- declarations that exist only in the TEST build of the library (libcwl_hooks.so, the same
+ * sources compiled with -DCWL_TEST_HOOKS).  The shipped libcwl.so has none of this.
+ */
+#ifndef CWL_TEST_HOOKS_H
+#define CWL_TEST_HOOKS_H
+
+#include "cwl.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Test hook for the failure path of cwl_apply and its variants.  Every device-side wait (mbarrier, H' flag, split-K
+ * counter) is bounded; when one runs out the CTA raises CWL_ERR_TIMEOUT in *status_word (bit 1 << CWL_ERR_TIMEOUT),
+ * drains its copies, frees its tensor memory and returns, so the context stays usable.  This call sets the limit
+ * (ns; <= 0 restores the default of 2 s) and, with withhold_publish != 0, makes the shrink never publish H', so that
+ * the waits on it run out.  Process-wide (two atomics). */
+void cwl_debug_set(int64_t wait_limit_ns, int32_t withhold_publish);
+
+/* Read-bandwidth ceiling of one decode-sized launch: 148 CTAs (one per SM) stream [ptr, ptr + bytes) once, each its
+ * slice, through a 192 KB shared-memory ring with contiguous 16 KB bulk copies, and drop the data.  No tensor-core
+ * work, no outputs.  Launched like the apply kernel (its set-up may overlap the tail of the launch ahead of it).
+ *   ptr  DEV, 128-byte aligned; bytes >= 148 * 16 KB (whole 16 KB pieces per CTA are read).
+ * Errors: INVALID_ARG, CUDA; a wait that runs out flags CWL_ERR_TIMEOUT in *status_word. */
+cwl_status cwl_probe_read(const void* ptr, size_t bytes, int32_t* status_word, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CWL_TEST_HOOKS_H */

@@ -6,6 +6,7 @@ been built, loading raises.  Function names mirror the C ABI declared in ``inclu
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes as C
 import os
 from typing import Optional, Sequence
@@ -22,8 +23,9 @@ STATUS = {0: "CWL_OK", 1: "CWL_ERR_INVALID_ARG", 2: "CWL_ERR_SHAPE", 3: "CWL_ERR
 EXPORTS = ["cwl_status_string", "cwl_version", "cwl_score_tokens", "cwl_score_tokens_mixed", "cwl_partition_workspace_bytes",
            "cwl_partition", "cwl_apply_workspace_bytes", "cwl_apply", "cwl_apply_grouped_workspace_bytes",
            "cwl_apply_grouped", "cwl_apply_plan", "cwl_stream_state_bytes", "cwl_stream_reset", "cwl_stream_step",
-           "cwl_apply_rows", "cwl_ladder_workspace_bytes", "cwl_ladder_build", "cwl_debug_set",
-           "cwl_apply_noalloc_scratch_need", "cwl_apply_noalloc", "cwl_prefetch_next", "cwl_apply_mode"]
+           "cwl_apply_rows", "cwl_ladder_workspace_bytes", "cwl_ladder_build",
+           "cwl_apply_noalloc_scratch_need", "cwl_apply_noalloc", "cwl_prefetch_next", "cwl_apply_mode",
+           "cwl_batch_align_workspace_bytes", "cwl_batch_align", "cwl_set_pair_budget"]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 WINDOW_CAUSAL, WINDOW_CENTRED = 0, 1
 
@@ -79,6 +81,8 @@ class CApplyPlanInfo(C.Structure):
 
 
 _lib = None
+_hooks_lib = None
+HOOKS_LIB_PATH = os.path.join(_HERE, "libcwl_hooks.so")
 
 
 def lib():
@@ -88,7 +92,33 @@ def lib():
         if not os.path.exists(LIB_PATH):
             raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2601_21109_b200.build` "
                                "(there is no fallback path)")
-        L = C.CDLL(LIB_PATH)
+        _lib = _declare(C.CDLL(LIB_PATH))
+    return _lib
+
+
+@contextlib.contextmanager
+def test_hooks():
+    """Routes every call of this module through the TEST build of the library (libcwl_hooks.so: the same sources
+    compiled with -DCWL_TEST_HOOKS, which adds cwl_debug_set) for the duration of the block."""
+    global _lib, _hooks_lib
+    if _hooks_lib is None:
+        if not os.path.exists(HOOKS_LIB_PATH):
+            raise RuntimeError(f"{HOOKS_LIB_PATH} is missing: run `python -m paper_2601_21109_b200.build`")
+        _hooks_lib = _declare(C.CDLL(HOOKS_LIB_PATH))
+        _hooks_lib.cwl_debug_set.restype = None
+        _hooks_lib.cwl_debug_set.argtypes = [C.c_int64, C.c_int32]
+    saved = lib()
+    _lib = _hooks_lib
+    try:
+        yield _hooks_lib
+    finally:
+        _hooks_lib.cwl_debug_set(0, 0)
+        _lib = saved
+
+
+def _declare(L):
+    """Argument and result types of every exported call."""
+    if True:
         L.cwl_status_string.restype = C.c_char_p
         L.cwl_status_string.argtypes = [C.c_int]
         L.cwl_version.restype = C.c_int
@@ -102,6 +132,11 @@ def lib():
         L.cwl_partition.restype = C.c_int
         L.cwl_partition.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(CPolicy), CChunkTable,
                                     C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        L.cwl_batch_align_workspace_bytes.restype = C.c_size_t
+        L.cwl_batch_align_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
+        L.cwl_batch_align.restype = C.c_int
+        L.cwl_batch_align.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(CPolicy), C.c_int32,
+                                      CChunkTable, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         L.cwl_apply_workspace_bytes.restype = C.c_size_t
         L.cwl_apply_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32]
         L.cwl_apply.restype = C.c_int
@@ -135,10 +170,10 @@ def lib():
         L.cwl_ladder_build.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
                                        C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_size_t, C.POINTER(C.c_int32), C.c_void_p]
+        L.cwl_set_pair_budget.restype = C.c_int
+        L.cwl_set_pair_budget.argtypes = [C.c_int32]
         L.cwl_prefetch_next.restype = C.c_int
         L.cwl_prefetch_next.argtypes = [C.c_void_p, C.c_size_t]
-        L.cwl_debug_set.restype = None
-        L.cwl_debug_set.argtypes = [C.c_int64, C.c_int32]
         L.cwl_apply_plan.restype = C.c_int
         L.cwl_apply_plan.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(CApplyPlanInfo)]
         L.cwl_apply_noalloc_scratch_need.restype = C.c_size_t
@@ -147,8 +182,7 @@ def lib():
         L.cwl_apply_noalloc.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
                                         C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                         CChunkTable, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
-        _lib = L
-    return _lib
+    return L
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
@@ -267,6 +301,27 @@ def cwl_partition(score: torch.Tensor, cu_seqlens: torch.Tensor, policy: CPolicy
                                                 table.c_struct(), _p(workspace), workspace.numel(),
                                                 _p(status_word), _stream_ptr(stream)))
     return table
+
+
+def cwl_batch_align(score: torch.Tensor, cu_seqlens: torch.Tensor, policy: CPolicy, n_buckets: int,
+                    table: Optional[DeviceChunkTable] = None, workspace: Optional[torch.Tensor] = None,
+                    status_word: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """Batch alignment: sequences bucketed by complexity percentile share their chunk joins.
+    Returns (table, bucket [n_seq] int32, order_pos [n_seq] int32), all on the device."""
+    assert score.is_cuda and score.dtype == torch.float32 and score.is_contiguous()
+    assert cu_seqlens.is_cuda and cu_seqlens.dtype == torch.int32 and cu_seqlens.is_contiguous()
+    T, n_seq = score.shape[0], cu_seqlens.shape[0] - 1
+    if table is None:
+        table = DeviceChunkTable(T // max(int(policy.min_len), 1) + n_seq + 1, score.device)
+    bucket = torch.empty(max(n_seq, 1), dtype=torch.int32, device=score.device)
+    order_pos = torch.empty(max(n_seq, 1), dtype=torch.int32, device=score.device)
+    if workspace is None:
+        workspace = torch.empty(max(16, int(lib().cwl_batch_align_workspace_bytes(T, n_seq, n_buckets))), dtype=torch.uint8,
+                                device=score.device)
+    _check("cwl_batch_align", lib().cwl_batch_align(_p(score), _p(cu_seqlens), n_seq, T, C.byref(policy), int(n_buckets),
+                                                    table.c_struct(), _p(bucket), _p(order_pos), _p(workspace),
+                                                    workspace.numel(), _p(status_word), _stream_ptr(stream)))
+    return table, bucket[:n_seq], order_pos[:n_seq]
 
 
 def cwl_apply_workspace_bytes(T: int, d_in: int, d_out: int, R: int) -> int:
@@ -424,18 +479,27 @@ def cwl_ladder_build(A: torch.Tensor, B: torch.Tensor, want_f32: bool = True,
     return out
 
 
-def cwl_prefetch_next(t: Optional[torch.Tensor]) -> None:
+def cwl_set_pair_budget(pairs: int) -> None:
+    """Apply calls of this thread plan for at most `pairs` CTA pairs from now on (0: the whole GPU)."""
+    _check("cwl_set_pair_budget", lib().cwl_set_pair_budget(int(pairs)))
+
+
+def cwl_prefetch_next(t: Optional[torch.Tensor], max_bytes: Optional[int] = None) -> None:
     """One-shot hint: the next apply call of this thread asks L2, while it drains, for the memory of `t` (the
-    weights the call after it will stream).  None withdraws a pending hint."""
+    weights the call after it will stream), or for its first `max_bytes` bytes.  None withdraws a pending hint."""
     if t is None:
         lib().cwl_prefetch_next(None, 0)
     else:
-        _check("cwl_prefetch_next", lib().cwl_prefetch_next(_p(t), t.numel() * t.element_size()))
+        n = t.numel() * t.element_size()
+        _check("cwl_prefetch_next", lib().cwl_prefetch_next(_p(t), n if max_bytes is None else min(n, int(max_bytes))))
 
 
 def cwl_debug_set(wait_limit_ns: int = 0, withhold_publish: bool = False) -> None:
-    """Test hook: device-side wait limit (<= 0: default) and whether the shrink withholds H' (timeout path)."""
-    lib().cwl_debug_set(int(wait_limit_ns), 1 if withhold_publish else 0)
+    """Test hook, inside ``with test_hooks():`` only: device-side wait limit (<= 0: default) and whether the shrink
+    withholds H' (timeout path)."""
+    if _lib is not _hooks_lib or _hooks_lib is None:
+        raise RuntimeError("cwl_debug_set exists in the test build only: call it inside `with binding.test_hooks():`")
+    _hooks_lib.cwl_debug_set(int(wait_limit_ns), 1 if withhold_publish else 0)
 
 
 def cwl_apply_noalloc(X: torch.Tensor, W: torch.Tensor, A: Optional[torch.Tensor], B: Optional[torch.Tensor],

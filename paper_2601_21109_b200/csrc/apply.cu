@@ -1245,6 +1245,13 @@ int max_pairs() {
   return n;
 }
 
+// Share of the GPU the calling host thread's apply calls plan for (cwl_set_pair_budget); 0 = all resident pairs.
+thread_local int t_pair_budget = 0;
+int pairs_now() {
+  const int all = max_pairs();
+  return t_pair_budget > 0 && t_pair_budget < all ? t_pair_budget : all;
+}
+
 // Launch epochs: 56 bits, starting from a per-process random value so that stale words of another process do not
 // match either; a word of arbitrary memory matches a given launch with probability 2^-56.
 unsigned long long next_epoch() {
@@ -1262,9 +1269,11 @@ unsigned long long next_epoch() {
 struct NextPrefetch { const unsigned char* ptr; unsigned long long bytes; };
 thread_local NextPrefetch t_next_prefetch = {nullptr, 0};
 
-// process-wide test hook state (cwl_debug_set)
-unsigned long long g_wait_limit_ns = kWaitLimitNs;
-int g_withhold_publish = 0;
+#ifdef CWL_TEST_HOOKS
+// process-wide test hook state (cwl_debug_set); only the test build of the library has it
+std::atomic<unsigned long long> g_wait_limit_ns{kWaitLimitNs};
+std::atomic<int> g_withhold_publish{0};
+#endif
 
 struct ApplyWorkspace { __nv_bfloat16* Hg; float* partial; float* sk_partial; unsigned long long* sync; size_t sync_bytes; };
 
@@ -1337,12 +1346,12 @@ cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* pr
   for (int j = 0; j < n_proj; ++j) d_out[j] = proj[j].d_out;
 
   ApplyWorkspace ws{nullptr, nullptr, nullptr, nullptr, 0};
-  Plan pl = make_plan(T, d_in, n_proj, d_out, Reff, max_pairs(), allow_split_k, scratch_limit);
+  Plan pl = make_plan(T, d_in, n_proj, d_out, Reff, pairs_now(), allow_split_k, scratch_limit);
   const size_t need = carve_apply(ws, static_cast<char*>(workspace), pl, T, Reff);
   const bool have_ws = workspace != nullptr && workspace_bytes >= need && (reinterpret_cast<uintptr_t>(workspace) & 255u) == 0;
   if (!have_ws && !adapter && pl.split_k > 1) {
     // the plain projection needs scratch only when its K loop is split; without a workspace it runs unsplit
-    pl = make_plan(T, d_in, n_proj, d_out, Reff, max_pairs(), false, scratch_limit);
+    pl = make_plan(T, d_in, n_proj, d_out, Reff, pairs_now(), false, scratch_limit);
   } else if (!have_ws && (adapter || pl.split_k > 1)) {
     return CWL_ERR_WORKSPACE;
   }
@@ -1369,7 +1378,11 @@ cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* pr
   p.Hg = ws.Hg; p.partial = ws.partial; p.sk_partial = ws.sk_partial;
   p.counters = ws.sync; p.flags = ws.sync + 2 * pl.n_m_pairs * n_proj; p.sk_counters = ws.sync + 4 * pl.n_m_pairs * n_proj;
   p.table = table; p.row_gates = row_gates; p.status_word = status_word;
-  p.wait_limit_ns = g_wait_limit_ns; p.withhold_publish = g_withhold_publish;
+#ifdef CWL_TEST_HOOKS
+  p.wait_limit_ns = g_wait_limit_ns.load(); p.withhold_publish = g_withhold_publish.load();
+#else
+  p.wait_limit_ns = kWaitLimitNs; p.withhold_publish = 0;
+#endif
   p.plan = pl;
   p.pf_ptr = hint.ptr; p.pf_bytes = hint.bytes;
 
@@ -1430,8 +1443,14 @@ cwl_status apply_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, co
 extern "C" size_t cwl_apply_workspace_bytes(int32_t T, int32_t d_in, int32_t d_out, int32_t R) {
   if (T <= 0 || d_in <= 0 || d_out <= 0 || R < 0) return 256;
   cwl::ApplyWorkspace w;
-  const cwl::Plan pl = cwl::make_plan(T, d_in, 1, &d_out, R, cwl::max_pairs(), true);
+  const cwl::Plan pl = cwl::make_plan(T, d_in, 1, &d_out, R, cwl::pairs_now(), true);
   return cwl::carve_apply(w, nullptr, pl, T, R);
+}
+
+extern "C" cwl_status cwl_set_pair_budget(int32_t pairs) {
+  if (pairs < 0) return CWL_ERR_INVALID_ARG;
+  cwl::t_pair_budget = pairs;
+  return CWL_OK;
 }
 
 extern "C" cwl_status cwl_prefetch_next(const void* ptr, size_t bytes) {
@@ -1444,10 +1463,12 @@ extern "C" cwl_status cwl_prefetch_next(const void* ptr, size_t bytes) {
   return CWL_OK;
 }
 
+#ifdef CWL_TEST_HOOKS
 extern "C" void cwl_debug_set(int64_t wait_limit_ns, int32_t withhold_publish) {
-  cwl::g_wait_limit_ns = wait_limit_ns > 0 ? (unsigned long long)wait_limit_ns : cwl::kWaitLimitNs;
-  cwl::g_withhold_publish = withhold_publish != 0 ? 1 : 0;
+  cwl::g_wait_limit_ns.store(wait_limit_ns > 0 ? (unsigned long long)wait_limit_ns : cwl::kWaitLimitNs);
+  cwl::g_withhold_publish.store(withhold_publish != 0 ? 1 : 0);
 }
+#endif
 
 extern "C" cwl_status cwl_apply_plan(int32_t T, int32_t d_in, int32_t d_out, int32_t R, int32_t pairs,
                                      cwl_apply_plan_info* out) {
@@ -1494,7 +1515,7 @@ extern "C" size_t cwl_apply_grouped_workspace_bytes(int32_t T, int32_t d_in, int
   int widths[CWL_MAX_GROUP];
   for (int j = 0; j < n_proj; ++j) { if (d_out[j] < 1) return 256; widths[j] = d_out[j]; }
   cwl::ApplyWorkspace w;
-  const cwl::Plan pl = cwl::make_plan(T, d_in, n_proj, widths, R, cwl::max_pairs(), true);
+  const cwl::Plan pl = cwl::make_plan(T, d_in, n_proj, widths, R, cwl::pairs_now(), true);
   return cwl::carve_apply(w, nullptr, pl, T, R);
 }
 
@@ -1553,7 +1574,7 @@ cwl_status noalloc_scratch(void** out) {
 extern "C" size_t cwl_apply_noalloc_scratch_need(int32_t T, int32_t d_in, int32_t d_out, int32_t R) {
   if (T <= 0 || d_in <= 0 || d_out <= 0 || R < 0) return 256;
   cwl::ApplyWorkspace w;
-  const cwl::Plan pl = cwl::make_plan(T, d_in, 1, &d_out, R, cwl::max_pairs(), false, CWL_NOALLOC_SCRATCH_BYTES);
+  const cwl::Plan pl = cwl::make_plan(T, d_in, 1, &d_out, R, cwl::pairs_now(), false, CWL_NOALLOC_SCRATCH_BYTES);
   return cwl::carve_apply(w, nullptr, pl, T, R);
 }
 

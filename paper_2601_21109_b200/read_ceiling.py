@@ -1,0 +1,67 @@
+"""Read-bandwidth ceiling of a decode-sized launch, measured with the test build's cwl_probe_read.
+
+    python -m paper_2601_21109_b200.read_ceiling [--mb 33.5 90.2 180.4 360.7] [--seconds 1.0]
+
+For every size: back-to-back launches (chained like the apply kernel's) rotate over enough distinct regions to
+exceed L2 several times, so every launch reads from HBM; CUDA events bracket the whole loop.  One launch = 148
+CTAs, each streaming its slice through a 192 KB shared-memory ring with 16 KB bulk copies and dropping the data.
+Prints microseconds per launch and GB/s; the figure for 90 MB (the bytes of one 4096 x 11008 bf16 projection) is
+what a decode launch could reach if its tensor-core work, hand-over and output stores cost nothing."""
+from __future__ import annotations
+
+import argparse
+import ctypes as C
+import json
+import math
+
+import torch
+
+from . import binding as cwl
+
+
+def measure(mb: float, seconds: float) -> dict:
+    n_bytes = int(mb * 1e6) // (148 * 16384) * (148 * 16384)
+    n_regions = max(4, int(math.ceil(600e6 / n_bytes)))            # >= 600 MB in rotation: several times L2
+    regions = [torch.empty(n_bytes, dtype=torch.uint8, device="cuda").fill_(i + 1) for i in range(n_regions)]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+    with cwl.test_hooks() as L:
+        L.cwl_probe_read.restype = C.c_int
+        L.cwl_probe_read.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+
+        def launch(i):
+            rc = L.cwl_probe_read(regions[i % n_regions].data_ptr(), n_bytes, status.data_ptr(), stream.cuda_stream)
+            if rc != 0:
+                raise RuntimeError(f"cwl_probe_read: status {rc}")
+        for i in range(2 * n_regions):
+            launch(i)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(20):
+            launch(i)
+        b.record()
+        torch.cuda.synchronize()
+        n = max(20, int(seconds * 1e3 / max(a.elapsed_time(b) / 20, 1e-3)))
+        a.record()
+        for i in range(n):
+            launch(i)
+        b.record()
+        torch.cuda.synchronize()
+    if int(status.item()) != 0:
+        raise RuntimeError(f"device status word {int(status.item()):#x}")
+    us = a.elapsed_time(b) * 1e3 / n
+    return {"mb": n_bytes / 1e6, "regions": n_regions, "launches": n, "us_per_launch": us, "gb_per_s": n_bytes / us / 1e3}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--mb", type=float, nargs="*", default=[33.6, 90.2, 180.4, 360.7])
+    ap.add_argument("--seconds", type=float, default=1.0)
+    args = ap.parse_args()
+    for mb in args.mb:
+        print(json.dumps(measure(mb, args.seconds)))
+
+
+if __name__ == "__main__":
+    main()

@@ -37,9 +37,9 @@ class HotPath:
 
     def __init__(self, w: Workload, device: str = "cuda", keep_host: bool = False, n_layers: int = 1,
                  grouped: bool = True, streaming: bool = False, share_weights: Optional["HotPath"] = None,
-                 prefetch: bool = True):
+                 prefetch_bytes: int = 0):
         self.grouped = grouped
-        self.prefetch = prefetch
+        self.prefetch_bytes = int(prefetch_bytes)    # decode: bytes of the next call's weights hinted to each call (0 = none)
         # decode with the token-by-token scheduler: every step the cached per-sequence state advances by one
         # token (the rows' scores) and the projections take the row gates it emits instead of a chunk table
         self.streaming = streaming
@@ -133,7 +133,7 @@ class HotPath:
     PREFETCH_MAX_T = 512
 
     def _next_weights(self, layer: int, i: int, next_layer: Optional[int]) -> Optional[torch.Tensor]:
-        if not self.prefetch or self.T >= self.PREFETCH_MAX_T:
+        if self.prefetch_bytes <= 0 or self.T >= self.PREFETCH_MAX_T:
             return None
         projs = self.layers[layer]
         if i + 1 < len(projs):
@@ -147,7 +147,7 @@ class HotPath:
             for i, p in enumerate(self.layers[layer]):
                 nxt = self._next_weights(layer, i, next_layer)
                 if nxt is not None:
-                    cwl.cwl_prefetch_next(nxt)
+                    cwl.cwl_prefetch_next(nxt, self.prefetch_bytes)
                 cwl.cwl_apply_rows(self.X[p.d_in], p.W, p.A, p.B, self.stream_state.gates, Y=p.Y,
                                    workspace=self.apply_ws, status_word=self.status)
             return
@@ -157,7 +157,7 @@ class HotPath:
             if len(group) == 1:
                 nxt = self._next_weights(layer, i, next_layer)
                 if nxt is not None:
-                    cwl.cwl_prefetch_next(nxt)
+                    cwl.cwl_prefetch_next(nxt, self.prefetch_bytes)
                 cwl.cwl_apply(self.X[p.d_in], p.W, None if dense else p.A, None if dense else p.B, tab,
                               self.policy.window, Y=p.Y, workspace=self.apply_ws, status_word=self.status)
             else:

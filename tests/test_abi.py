@@ -33,6 +33,15 @@ def test_library_exports_every_declared_symbol(lib_path):
         assert hasattr(lib, name), name
 
 
+def test_the_test_hook_exists_in_the_test_build_only(lib_path):
+    from paper_2601_21109_b200 import build
+    assert not hasattr(ctypes.CDLL(lib_path), "cwl_debug_set")
+    hooks = ctypes.CDLL(build.LIB_HOOKS)
+    assert hasattr(hooks, "cwl_debug_set")
+    for name in declared_functions():                        # and everything else as well
+        assert hasattr(hooks, name), name
+
+
 def test_binding_covers_the_header(lib_path):
     from paper_2601_21109_b200 import binding
     assert sorted(binding.EXPORTS) == declared_functions()

@@ -1,4 +1,5 @@
-"""The failure path of cwl_apply without a device fault: with the test hook the shrink never publishes H', every
+"""The failure path of cwl_apply without a device fault: with the test hook (test build of the library only) the
+shrink never publishes H', every
 wait on it runs out after a short limit, the kernel reports CWL_ERR_TIMEOUT in the status word and returns, and
 the very next ordinary call on the same context is correct."""
 import numpy as np
@@ -23,7 +24,7 @@ def test_withheld_publication_times_out_and_the_context_stays_usable():
                flags=np.array([1, 0], np.int32), rung=np.zeros(2, np.int32), n_chunks=2)
     args = (dev_bf16(X), dev_bf16(W), dev_bf16(A), dev_bf16(B), dev_table(tab), 8)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    try:
+    with cwl.test_hooks():                                                       # the test build of the library
         cwl.cwl_debug_set(wait_limit_ns=20_000_000, withhold_publish=True)      # 20 ms
         start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         start.record()
@@ -32,8 +33,6 @@ def test_withheld_publication_times_out_and_the_context_stays_usable():
         torch.cuda.synchronize()                                                 # returns: nothing hangs
         assert int(status.item()) & (1 << CWL_ERR_TIMEOUT)
         assert start.elapsed_time(end) < 2000.0                                  # a few wait limits, not seconds
-    finally:
-        cwl.cwl_debug_set(0, False)
     status.zero_()
     Y = cwl.cwl_apply(*args, status_word=status)
     torch.cuda.synchronize()
