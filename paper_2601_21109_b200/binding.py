@@ -355,9 +355,8 @@ def cwl_apply(X: torch.Tensor, W: torch.Tensor, A: Optional[torch.Tensor], B: Op
         R = A.shape[1]
     if Y is None:
         Y = torch.empty(T, d_out, dtype=torch.bfloat16, device=X.device)
-    need = cwl_apply_workspace_bytes(T, d_in, d_out, R)
     if workspace is None:
-        workspace = torch.empty(need, dtype=torch.uint8, device=X.device)
+        workspace = torch.empty(cwl_apply_workspace_bytes(T, d_in, d_out, R), dtype=torch.uint8, device=X.device)
     ct = table.c_struct() if table is not None else CChunkTable(None, None, None, None, None, None, 0)
     if centred:
         _check("cwl_apply_mode", lib().cwl_apply_mode(_p(X), X.stride(0), _p(W), W.stride(0),

@@ -37,7 +37,7 @@ class HotPath:
 
     def __init__(self, w: Workload, device: str = "cuda", keep_host: bool = False, n_layers: int = 1,
                  grouped: bool = True, streaming: bool = False, share_weights: Optional["HotPath"] = None,
-                 prefetch_bytes: int = 0):
+                 prefetch_bytes: int = 0, concurrent: bool = True):
         self.grouped = grouped
         self.prefetch_bytes = int(prefetch_bytes)    # decode: bytes of the next call's weights hinted to each call (0 = none)
         # decode with the token-by-token scheduler: every step the cached per-sequence state advances by one
@@ -84,6 +84,22 @@ class HotPath:
                 ws_bytes = max(ws_bytes, cwl.cwl_apply_grouped_workspace_bytes(
                     w.T, group[0].d_in, [q.d_out for q in group], w.R))
         self.apply_ws = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
+        # Decode-sized steps: the projections of a step are independent calls, and each spends a large share of its
+        # launch setting up and draining.  They are issued side by side on `lanes` streams, each call planned for its
+        # share of the CTA pairs (cwl_set_pair_budget), so that one call's set-up and drain overlap the other's main
+        # loop.  Every lane has a workspace of its own.
+        self.lanes = 2 if (concurrent and w.T < self.GROUP_MIN_T and len(w.projections) >= 2) else 1
+        if self.lanes > 1:
+            self.lane_budget = [self.RESIDENT_PAIRS // self.lanes] * self.lanes
+            self.lane_streams = [torch.cuda.Stream(device=device) for _ in range(self.lanes)]
+            self.lane_ws = []
+            for b in self.lane_budget:
+                cwl.cwl_set_pair_budget(b)
+                n = max(cwl.cwl_apply_workspace_bytes(w.T, p.d_in, p.d_out, w.R) for p in w.projections)
+                self.lane_ws.append(torch.empty(n, dtype=torch.uint8, device=device))
+            cwl.cwl_set_pair_budget(0)
+            self.fork_event = torch.cuda.Event()
+            self.join_events = [torch.cuda.Event() for _ in range(self.lanes)]
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
         self.cpolicy = policy_struct(w.policy)
         self.stream_state = cwl.DeviceStream(w.T, self.cpolicy, device) if streaming else None
@@ -111,6 +127,7 @@ class HotPath:
     # gain 9 % at T = 8192.  Below GROUP_MIN_T a call is decode-sized: separate calls, whose K loop is split.
     GROUPS = ((("q", "k", "v"), 4096), (("gate", "up"), 512))    # (members, smallest T at which they are grouped)
     GROUP_MIN_T = 512
+    RESIDENT_PAIRS = 74          # CTA pairs a B200 holds (148 SMs)
 
     def launch_groups(self, layer: int = 0) -> List[List[DeviceProjection]]:
         projs = self.layers[layer]
@@ -143,7 +160,30 @@ class HotPath:
 
     def apply_step(self, table: Optional[cwl.DeviceChunkTable] = None, dense: bool = False, layer: int = 0,
                    next_layer: Optional[int] = None) -> None:
-        if self.streaming and table is None and not dense:
+        rows = self.streaming and table is None and not dense
+        tab = table if table is not None else self.table
+        if self.lanes > 1:
+            # fork: the lanes start where the current stream stands; join: it continues once every lane is done
+            main = torch.cuda.current_stream()
+            self.fork_event.record(main)
+            for st in self.lane_streams:
+                st.wait_event(self.fork_event)
+            for i, p in enumerate(self.layers[layer]):
+                j = i % self.lanes
+                cwl.cwl_set_pair_budget(self.lane_budget[j])
+                if rows:
+                    cwl.cwl_apply_rows(self.X[p.d_in], p.W, p.A, p.B, self.stream_state.gates, Y=p.Y,
+                                       workspace=self.lane_ws[j], status_word=self.status, stream=self.lane_streams[j])
+                else:
+                    cwl.cwl_apply(self.X[p.d_in], p.W, None if dense else p.A, None if dense else p.B, tab,
+                                  self.policy.window, Y=p.Y, workspace=self.lane_ws[j], status_word=self.status,
+                                  stream=self.lane_streams[j])
+            cwl.cwl_set_pair_budget(0)
+            for ev, st in zip(self.join_events, self.lane_streams):
+                ev.record(st)
+                main.wait_event(ev)
+            return
+        if rows:
             for i, p in enumerate(self.layers[layer]):
                 nxt = self._next_weights(layer, i, next_layer)
                 if nxt is not None:
@@ -151,7 +191,6 @@ class HotPath:
                 cwl.cwl_apply_rows(self.X[p.d_in], p.W, p.A, p.B, self.stream_state.gates, Y=p.Y,
                                    workspace=self.apply_ws, status_word=self.status)
             return
-        tab = table if table is not None else self.table
         for i, group in enumerate(self.launch_groups(layer)):
             p = group[0]
             if len(group) == 1:

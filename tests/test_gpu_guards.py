@@ -118,3 +118,27 @@ def test_score_and_partition_write_exactly_their_outputs():
     assert int(status.item()) == 0 and 0 < n <= tab.capacity
     assert bool((tab.offsets[n + 1:] == -99).all()) and bool((tab.rank[n:] == -99).all()) and bool((tab.flags[n:] == -99).all())
     assert int(tab.offsets[0]) == 0 and int(tab.offsets[n]) == T
+
+
+@pytest.mark.parametrize("budget", [37, 26, 9, 1])
+def test_a_call_planned_for_a_share_of_the_gpu_stays_inside_its_output_and_matches_the_full_plan(budget):
+    # cwl_set_pair_budget changes the plan (tile widths, K split, who computes the shrink), never the result
+    T, d_in, d_out, R = 200, 2048, 1552, 64
+    X, (W,), (A,), (B,) = operands(77, T, d_in, [d_out], R)
+    tab = table(T, R)
+    want = cwl.cwl_apply(X, W, A, B, tab, 8)
+    buf, Y = guarded(T, d_out)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    try:
+        cwl.cwl_set_pair_budget(budget)
+        cwl.cwl_apply(X, W, A, B, tab, 8, Y=Y, status_word=status)
+    finally:
+        cwl.cwl_set_pair_budget(0)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    check_guards(buf, T, d_out)
+    # the same products summed in another order: fp32 rounding differences only, at most one bf16 ulp after rounding
+    a, b = Y.float(), want.float()
+    assert float((a - b).abs().max()) <= float(b.abs().max()) * 2.0 ** -7
+    with pytest.raises(cwl.CwlError):
+        cwl.cwl_set_pair_budget(-1)
