@@ -422,6 +422,22 @@ def measure(name: str, args, steps: int, warmup: int, world: int, rank: int, loc
         torch.cuda.synchronize()
         apply_ms = sum(x.elapsed_time(y) for x, y in ev) / n2
 
+    # ---- decode with a fixed table: the same steps with the lanes left running (no join between steps; each lane keeps
+    # its order and the region ends with a join).  The steps of this workload do not depend on one another, so this is a
+    # legal schedule; the headline figure above keeps the join after every step.
+    free_ms = None
+    if decode and not streaming and hp.lanes > 1 and not args.lean:
+        n3 = max(steps, int(math.ceil(0.5e3 / max(ms_per_step, 1e-3))))
+        x, y = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        x.record(stream)
+        for i in range(n3):
+            hp.apply_step(layer=i % n_layers, join=False, fork=(i == 0))
+        hp.join_lanes()
+        y.record(stream)
+        torch.cuda.synchronize()
+        free_ms = x.elapsed_time(y) / n3
+
     # ---- comparison runs through the same kernels: static full-rank LoRA and the dense floor ---
     static_ms = dense_ms = chunk_only_ms = None
     if not args.lean:
@@ -522,7 +538,8 @@ def measure(name: str, args, steps: int, warmup: int, world: int, rank: int, loc
            "config": dict(config_dict(name, w, n_layers, world, not args.no_group)),
            "n_chunks": int(table["n_chunks"]) if table is not None else None,
            "tflops": f_alg * n_steps * world / (ms_total * 1e-3) / 1e12,
-           "apply_ms_per_step": apply_ms, "apply_only_loop_ms": chunk_only_ms,
+           "apply_ms_per_step": apply_ms, "apply_only_loop_ms": chunk_only_ms, "lanes": hp.lanes,
+           "free_running_lanes_ms_per_step": free_ms,
            "static_lora_apply_ms": static_ms, "dense_floor_apply_ms": dense_ms,
            "clocks": clocks, "gpu_launches": hp.launches_per_step(stack) * n_steps, "roofline": roof}
     if e2e is not None:

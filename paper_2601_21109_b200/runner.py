@@ -158,16 +158,29 @@ class HotPath:
         nl = (layer + 1) % len(self.layers) if next_layer is None else next_layer
         return self.layers[nl][0].W
 
+    def join_lanes(self) -> None:
+        """The current stream continues once every lane has finished what it was given."""
+        if self.lanes > 1:
+            main = torch.cuda.current_stream()
+            for ev, st in zip(self.join_events, self.lane_streams):
+                ev.record(st)
+                main.wait_event(ev)
+
     def apply_step(self, table: Optional[cwl.DeviceChunkTable] = None, dense: bool = False, layer: int = 0,
-                   next_layer: Optional[int] = None) -> None:
+                   next_layer: Optional[int] = None, join: bool = True, fork: bool = True) -> None:
+        """The adapted projections of one layer.  With lanes, `join=False` leaves the lanes running on their own
+        streams (each lane keeps its own order; call join_lanes() before anything reads the outputs) and `fork=False`
+        does not make them wait for the current stream again: steps whose projections do not depend on one another
+        can then follow one another without draining the GPU in between."""
         rows = self.streaming and table is None and not dense
         tab = table if table is not None else self.table
         if self.lanes > 1:
             # fork: the lanes start where the current stream stands; join: it continues once every lane is done
-            main = torch.cuda.current_stream()
-            self.fork_event.record(main)
-            for st in self.lane_streams:
-                st.wait_event(self.fork_event)
+            if fork:
+                main = torch.cuda.current_stream()
+                self.fork_event.record(main)
+                for st in self.lane_streams:
+                    st.wait_event(self.fork_event)
             for i, p in enumerate(self.layers[layer]):
                 j = i % self.lanes
                 cwl.cwl_set_pair_budget(self.lane_budget[j])
@@ -179,9 +192,8 @@ class HotPath:
                                   self.policy.window, Y=p.Y, workspace=self.lane_ws[j], status_word=self.status,
                                   stream=self.lane_streams[j])
             cwl.cwl_set_pair_budget(0)
-            for ev, st in zip(self.join_events, self.lane_streams):
-                ev.record(st)
-                main.wait_event(ev)
+            if join:
+                self.join_lanes()
             return
         if rows:
             for i, p in enumerate(self.layers[layer]):

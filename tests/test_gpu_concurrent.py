@@ -20,9 +20,11 @@ def problem(seed, T, d_in, d_out, R):
                 A=wl.normal_bf16(rng, (d_in, R), d_in ** -0.5), B=wl.normal_bf16(rng, (R, d_out), R ** -0.5))
     cuts = sorted(rng.choice(np.arange(64, T - 64, 16), size=5, replace=False).tolist())
     n = len(cuts) + 1
-    tab = dict(offsets=np.array([0] + cuts + [T], np.int32), rank=rng.choice([8, 16, 32, 64], n).astype(np.int32),
-               scale=rng.choice([4.0, 2.0, 1.0, 0.5], n).astype(np.float32), flags=np.array([1] + [0] * (n - 1), np.int32),
-               rung=np.zeros(n, np.int32), n_chunks=n)
+    rank = rng.choice([8, 16, 32, 64], n).astype(np.int32)
+    # scale = alpha / rank as the ladder sets it: the gated shrink output is a bf16 tensor-core operand, so its rounding
+    # (2^-9 relative) scales with the adapter term, which a large scale on a large rank would blow up beyond the 3e-2 gate
+    tab = dict(offsets=np.array([0] + cuts + [T], np.int32), rank=rank, scale=(32.0 / rank).astype(np.float32),
+               flags=np.array([1] + [0] * (n - 1), np.int32), rung=np.zeros(n, np.int32), n_chunks=n)
     return host, tab
 
 
