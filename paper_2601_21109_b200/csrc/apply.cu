@@ -63,6 +63,10 @@ constexpr int kABytes = BM * BK * 2;          // 16 KB: this CTA's 128 rows of t
 constexpr int kBoxBytes = kBoxCols * BK * 2;  // 8 KB
 constexpr int kMaxStages = 8;
 constexpr int kRingBytes = 192 * 1024;
+// A launch whose tiles split their K loop never stages whole output tiles, so its epilogue needs the row gates only:
+// the operand ring takes the room (one more 40 KB stage in flight for 336- and 384-wide decode tiles).
+constexpr int kRingBytesSplit = 216 * 1024;
+constexpr int kOutBytesSplit = 8 * 1024;
 constexpr int kOutBufBytes = 4096;  // per epilogue warp: 32 rows x 64 bf16 columns staged for row-contiguous stores
 constexpr int kThreads = 320;       // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: epilogue
 constexpr int kEpiThreads = 256;
@@ -449,7 +453,8 @@ struct SmemLayout {
   static constexpr int kMiscBytes = 32;              // TMEM base, abort flag, epilogue broadcast words
   static constexpr int kTotal = kRingBytes + kOutBytes + kBarBytes + kMiscBytes + 1024;  // + alignment slack
 };
-static_assert(BM * sizeof(RowGate) <= SmemLayout::kOutBytes, "row gates must fit the staging area");
+static_assert(BM * sizeof(RowGate) <= SmemLayout::kOutBytes && BM * sizeof(RowGate) <= kOutBytesSplit, "row gates must fit the staging area");
+static_assert(kRingBytesSplit + kOutBytesSplit == kRingBytes + SmemLayout::kOutBytes, "both instantiations use the same amount of shared memory");
 static_assert(SmemLayout::kTotal <= 227 * 1024, "shared memory budget");
 
 // Two instantiations: kSplitK = false for plans whose tiles keep their whole K loop (the epilogue stores whole
@@ -469,19 +474,21 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;     // swizzled tiles need 1024-byte alignment
   uint8_t* base_ptr = smem_raw + (base - raw);
-  const uint32_t out_bufs = base + kRingBytes;      // per-warp staging buffers of the epilogue
-  const uint32_t bars = out_bufs + L::kOutBytes;
+  constexpr int kRing = kSplitK ? kRingBytesSplit : kRingBytes;
+  constexpr int kOut = kSplitK ? kOutBytesSplit : L::kOutBytes;
+  const uint32_t out_bufs = base + kRing;           // per-warp staging buffers of the epilogue
+  const uint32_t bars = out_bufs + kOut;
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
   const uint32_t acc_full_bar = bars + 8u * (2 * kMaxStages);
   const uint32_t acc_empty_bar = bars + 8u * (2 * kMaxStages + 1);
   const uint32_t fix_bar = bars + 8u * (2 * kMaxStages + 2);   // split-K: the others' partial sums have landed
-  uint8_t* misc = base_ptr + kRingBytes + L::kOutBytes + L::kBarBytes;
+  uint8_t* misc = base_ptr + kRing + kOut + L::kBarBytes;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
   volatile int* epi_go = reinterpret_cast<volatile int*>(misc + 8);     // epilogue: proceed with this item?
   volatile int* epi_last = reinterpret_cast<volatile int*>(misc + 12);  // epilogue: this CTA finalises the row tile
-  RowGate* gates = reinterpret_cast<RowGate*>(base_ptr + kRingBytes);
+  RowGate* gates = reinterpret_cast<RowGate*>(base_ptr + kRing);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair (issues the MMAs)
@@ -605,38 +612,64 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    // One thread issues every MMA of the pair, so the instructions it executes per K block are on the critical path
+    // of narrow (decode-sized) tiles, whose tensor-core time per block is short: device timestamps showed 0.47 us from
+    // "operands landed" to "commit issued" for eight MMAs, more than the MMAs themselves take.  The loop therefore
+    // keeps running shared-memory descriptors (one 64-bit add per ring slot and per K step instead of rebuilding
+    // them), takes the common case of a full 64-deep block through an unrolled path, and works the K extent of the
+    // last block of each phase out once per item.
     if (lane == 0 && rank == 0) {
       uint32_t local = 0;
       uint32_t s = 0, ph = 0;   // ring slot and phase parity, kept incrementally
       bool ok = true;
       Item item;
+      // descriptors of ring slot 0; a slot is stage_bytes further on (the address field counts 16-byte units and the
+      // whole ring lies below 256 KB, so adding to the 64-bit descriptor never carries out of the field)
+      const uint64_t desc_a0 = make_smem_desc(base, 16, 1024);
+      const uint64_t desc_b0 = make_smem_desc(base + kABytes, kBoxBytes, 1024);
+      const uint64_t desc_slot = (uint64_t)(stage_bytes >> 4);
+      constexpr uint64_t kStepA = (UMMA_K * 2) >> 4;        // one K step further in a K-major tile
+      constexpr uint64_t kStepB = (UMMA_K * 128) >> 4;      // ... in an N-major box
+      uint64_t da = desc_a0, db = desc_b0;
       for (int i = 0; ok && get_item(i, pair, sh_begin, p, item); ++i, ++local) {
         const uint32_t idesc_a = make_idesc(2 * BM, item.wa);
         const uint32_t idesc_b = make_idesc(2 * BM, item.wb > 0 ? item.wb : 16);
-        const uint32_t sb_off_b = (uint32_t)boxes_for(item.wa >> 1) * kBoxBytes;
+        const uint64_t second = (uint64_t)((uint32_t)boxes_for(item.wa >> 1) * kBoxBytes >> 4);   // second MMA's boxes
+        const bool two = item.wb > 0;
         if (!mbar_wait(acc_empty_bar, (local & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const int n_blk = item.n_blk0 + item.n_blk1;
+        // K steps of the last block of the d_in phase (if this item holds the end of d_in) and of the R phase
+        const int tail0 = (item.kb0 + item.n_blk0 == pl.nkb0 && (p.d_in & (BK - 1)) != 0) ? (p.d_in & (BK - 1)) / UMMA_K : BK / UMMA_K;
+        const int tail1 = (p.R & (BK - 1)) != 0 ? (p.R & (BK - 1)) / UMMA_K : BK / UMMA_K;
         for (int b = 0; b < n_blk; ++b) {
           if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const bool phase1 = b >= item.n_blk0;
-          const int k = phase1 ? (b - item.n_blk0) * BK : (item.kb0 + b) * BK;
-          const int k_left = (phase1 ? p.R : p.d_in) - k;          // multiple of 16
-          const int k_steps = k_left >= BK ? BK / UMMA_K : k_left / UMMA_K;
-          const uint32_t sa = base + s * stage_bytes, sb = sa + kABytes;
-          for (int kk = 0; kk < k_steps; ++kk) {
-            const uint32_t acc_flag = (b | kk) != 0 ? 1u : 0u;
-            const uint64_t da = make_smem_desc(sa + kk * (UMMA_K * 2), 16, 1024);
-            const uint64_t db = make_smem_desc(sb + kk * (UMMA_K * 128), kBoxBytes, 1024);
-            umma_bf16_pair(tmem_base, da, db, idesc_a, acc_flag);
-            if (item.wb > 0) {
-              const uint64_t db2 = make_smem_desc(sb + sb_off_b + kk * (UMMA_K * 128), kBoxBytes, 1024);
-              umma_bf16_pair(tmem_base + kMmaN, da, db2, idesc_b, acc_flag);
+          int k_steps = BK / UMMA_K;
+          if (b == item.n_blk0 - 1) k_steps = tail0;
+          else if (b == n_blk - 1 && item.n_blk1 > 0) k_steps = tail1;
+          const uint32_t acc0 = b != 0 ? 1u : 0u;
+          if (k_steps == BK / UMMA_K) {
+            if (two) {
+#pragma unroll
+              for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+                umma_bf16_pair(tmem_base, da + kk * kStepA, db + kk * kStepB, idesc_a, kk ? 1u : acc0);
+                umma_bf16_pair(tmem_base + kMmaN, da + kk * kStepA, db + second + kk * kStepB, idesc_b, kk ? 1u : acc0);
+              }
+            } else {
+#pragma unroll
+              for (int kk = 0; kk < BK / UMMA_K; ++kk)
+                umma_bf16_pair(tmem_base, da + kk * kStepA, db + kk * kStepB, idesc_a, kk ? 1u : acc0);
+            }
+          } else {
+            for (int kk = 0; kk < k_steps; ++kk) {
+              umma_bf16_pair(tmem_base, da + kk * kStepA, db + kk * kStepB, idesc_a, kk ? 1u : acc0);
+              if (two) umma_bf16_pair(tmem_base + kMmaN, da + kk * kStepA, db + second + kk * kStepB, idesc_b, kk ? 1u : acc0);
             }
           }
           umma_commit_pair(empty_bar(s));            // frees the stage in both CTAs once these MMAs have read it
-          if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
+          if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; da = desc_a0; db = desc_b0; }
+          else { da += desc_slot; db += desc_slot; }
         }
         if (ok) umma_commit_pair(acc_full_bar);      // accumulator complete, both CTAs
       }
@@ -770,7 +803,7 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
         // dependent loads per thread.
         const uint32_t seg_bytes = (uint32_t)(c_hi - c_lo) * (BM * 4);          // one contributor's run
         const uint32_t land = ((uint32_t)(BM * pitch) + 1023u) & ~1023u;        // offset of the landing zone in the ring
-        const bool landed = c_hi > c_lo && land + (uint32_t)(pl.split_k - 1) * seg_bytes <= (uint32_t)kRingBytes;
+        const bool landed = c_hi > c_lo && land + (uint32_t)(pl.split_k - 1) * seg_bytes <= (uint32_t)kRing;
         if (epi_tid == 0) {
           __threadfence();                           // device-wide release of the CTA's partial (cumulative over the barrier)
           sync_arrive(counter, p.epoch);
@@ -1068,7 +1101,7 @@ Plan search_plan(int T, int d_in, int n_proj, const int* d_out, int R, int pairs
   pl.boxes = tile_boxes(pl.w0);
   if (pl.n_narrow > 0 && tile_boxes(pl.w1) > pl.boxes) pl.boxes = tile_boxes(pl.w1);
   if (R > 0 && boxes_for(R / 2) > pl.boxes) pl.boxes = boxes_for(R / 2);
-  pl.stages = kRingBytes / (kABytes + pl.boxes * kBoxBytes);
+  pl.stages = (pl.split_k > 1 ? kRingBytesSplit : kRingBytes) / (kABytes + pl.boxes * kBoxBytes);
   if (pl.stages > kMaxStages) pl.stages = kMaxStages;
 
   // ---- shrink: how finely d_in is split and who does the items.  Items go, one at a time, to the pair with
