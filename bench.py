@@ -11,7 +11,7 @@ workloads (single-sequence prefill, packed ragged prefill, decode with a fixed t
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
                     [--workload cfg5|cfg2|cfg3|cfg4|cfg4_stream|cfg1] [--layers L] [--min-seconds S]
-                    [--no-configs] [--no-group] [--no-concurrent] [--prefetch-mb M] [--lean]
+                    [--no-configs] [--no-group] [--decode-mode batch|lanes|serial] [--prefetch-mb M] [--lean]
 
 Every timed region lasts at least --min-seconds of device time: the block of K steps is repeated (`inner_repeats`)
 until it does, and ms_per_step is the mean over all K x repeats steps (median and min per block are beside it).
@@ -334,7 +334,7 @@ def measure(name: str, args, steps: int, warmup: int, world: int, rank: int, loc
     decode = name in ("cfg4", "cfg4_stream")
     streaming = name == "cfg4_stream"
     hp = HotPath(w, n_layers=n_layers, grouped=not args.no_group, streaming=streaming, prefetch_bytes=int(args.prefetch_mb * 1e6),
-                 concurrent=not args.no_concurrent)
+                 decode_mode=args.decode_mode)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -538,7 +538,7 @@ def measure(name: str, args, steps: int, warmup: int, world: int, rank: int, loc
            "config": dict(config_dict(name, w, n_layers, world, not args.no_group)),
            "n_chunks": int(table["n_chunks"]) if table is not None else None,
            "tflops": f_alg * n_steps * world / (ms_total * 1e-3) / 1e12,
-           "apply_ms_per_step": apply_ms, "apply_only_loop_ms": chunk_only_ms, "lanes": hp.lanes,
+           "apply_ms_per_step": apply_ms, "apply_only_loop_ms": chunk_only_ms, "decode_mode": hp.decode_mode if decode else None,
            "free_running_lanes_ms_per_step": free_ms,
            "static_lora_apply_ms": static_ms, "dense_floor_apply_ms": dense_ms,
            "clocks": clocks, "gpu_launches": hp.launches_per_step(stack) * n_steps, "roofline": roof}
@@ -630,8 +630,9 @@ def main():
     ap.add_argument("--no-configs", action="store_true", help="headline workload only: no `configs` block")
     ap.add_argument("--no-group", action="store_true",
                     help="one cwl_apply launch per projection instead of grouped launches for q,k,v and gate,up")
-    ap.add_argument("--no-concurrent", action="store_true",
-                    help="decode: the projections of a step one after the other on one stream, each planned for the whole GPU")
+    ap.add_argument("--decode-mode", default="batch", choices=["batch", "lanes", "serial"],
+                    help="decode: the step's projections as one batch launch (default), side by side on two streams, or one "
+                         "after the other on one stream, each planned for the whole GPU")
     ap.add_argument("--prefetch-mb", type=float, default=0.0,
                     help="decode: tell each call to pull this many MB of the next call's weights towards L2 while it drains (0: off)")
     ap.add_argument("--lean", action="store_true",

@@ -219,6 +219,30 @@ cwl_status cwl_apply_grouped(const void* X, int64_t ldx, const cwl_projection* p
                              int32_t T, int32_t d_in, int32_t R, cwl_chunk_table table, int32_t window,
                              void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream);
 
+/* Several INDEPENDENT adapted projections in one launch (Sec. III-F: the adapter sits on every attention and MLP
+ * projection; the projections of a decode step whose inputs are ready do not depend on one another).  Unlike
+ * cwl_apply_grouped the projections need not read the same rows: every item has its own X, d_in, W, A, B, Y, d_out;
+ * T, R, the chunk table (or the row gates) and the window are shared.  The CTA pairs are shared out among the items in
+ * proportion to the bytes of their weights and every item is planned and run exactly as a cwl_apply call on that many
+ * pairs would be; sharing one launch, the set-up and the drain of one item overlap the main loops of the others, and
+ * consecutive batch launches chain like any other launch.  Meant for decode-sized T, where set-up and drain are a
+ * large share of a launch.
+ *   items       HOST array of n descriptors (1 <= n <= CWL_MAX_BATCH), copied at call time; pointers inside are DEV.
+ *               An item with A == NULL or B == NULL computes X W only.
+ *   gates       DEV cwl_row_gate [T] (declared below) or NULL; when set, the rows' descriptors replace the chunk table
+ *   workspace   DEV, cwl_apply_batch_workspace_bytes(T, n, d_in[], d_out[], R) bytes, 256-byte aligned
+ * Results equal those of n cwl_apply / cwl_apply_rows calls up to the order of fp32 sums.  Shape rules and errors as
+ * for cwl_apply; UNSUPPORTED when fewer CTA pairs than items are available (cwl_set_pair_budget). */
+#define CWL_MAX_BATCH 4
+typedef struct {
+  const void* X; int64_t ldx; int32_t d_in;     /* DEV bf16 [T, d_in] */
+  const void* W; int64_t ldw;                   /* DEV bf16 [d_in, d_out] */
+  const void* A; int64_t lda;                   /* DEV bf16 [d_in, R] or NULL */
+  const void* B; int64_t ldb;                   /* DEV bf16 [R, d_out] or NULL */
+  void*       Y; int64_t ldy; int32_t d_out;    /* DEV bf16 [T, d_out] */
+} cwl_batch_item;
+size_t     cwl_apply_batch_workspace_bytes(int32_t T, int32_t n, const int32_t* d_in, const int32_t* d_out, int32_t R);
+
 /* Decode-time scheduler (Sec. III-A, III-B, III-F: scores arrive as tokens stream in, tokens are grouped as they
  * arrive, and the scheduler keeps its state from step to step): every step brings one new token per sequence.  The paper names the constraints only; the rule here is
  * causal.  Per sequence the state holds the open chunk's length and the rung it was opened on, the rung of the chunk
@@ -257,6 +281,11 @@ cwl_status cwl_apply_rows(const void* X, int64_t ldx, const void* W, int64_t ldw
                           int32_t T, int32_t d_in, int32_t d_out, int32_t R,
                           const cwl_row_gate* gates, void* Y, int64_t ldy,
                           void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream);
+
+/* cwl_apply_batch: see cwl_batch_item above (declared here because it takes row gates). */
+cwl_status cwl_apply_batch(const cwl_batch_item* items, int32_t n, int32_t T, int32_t R,
+                           cwl_chunk_table table, const cwl_row_gate* gates, int32_t window,
+                           void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream);
 
 /* Offline construction of the rank ladder (Sec. III-C: the ladder comes from a one-off singular value decomposition
  * of the trained adapter): re-factorises a

@@ -25,9 +25,11 @@ EXPORTS = ["cwl_status_string", "cwl_version", "cwl_score_tokens", "cwl_score_to
            "cwl_apply_grouped", "cwl_apply_plan", "cwl_stream_state_bytes", "cwl_stream_reset", "cwl_stream_step",
            "cwl_apply_rows", "cwl_ladder_workspace_bytes", "cwl_ladder_build",
            "cwl_apply_noalloc_scratch_need", "cwl_apply_noalloc", "cwl_prefetch_next", "cwl_apply_mode",
-           "cwl_batch_align_workspace_bytes", "cwl_batch_align", "cwl_set_pair_budget"]
+           "cwl_batch_align_workspace_bytes", "cwl_batch_align", "cwl_set_pair_budget",
+           "cwl_apply_batch_workspace_bytes", "cwl_apply_batch"]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 WINDOW_CAUSAL, WINDOW_CENTRED = 0, 1
+MAX_BATCH = 4
 
 
 class CwlError(RuntimeError):
@@ -65,6 +67,12 @@ ROW_GATE_BYTES = C.sizeof(CRowGate)     # 28: gates live in a uint8 tensor of [n
 
 class CProjection(C.Structure):
     _fields_ = [("W", C.c_void_p), ("ldw", C.c_int64), ("A", C.c_void_p), ("lda", C.c_int64),
+                ("B", C.c_void_p), ("ldb", C.c_int64), ("Y", C.c_void_p), ("ldy", C.c_int64), ("d_out", C.c_int32)]
+
+
+class CBatchItem(C.Structure):
+    _fields_ = [("X", C.c_void_p), ("ldx", C.c_int64), ("d_in", C.c_int32),
+                ("W", C.c_void_p), ("ldw", C.c_int64), ("A", C.c_void_p), ("lda", C.c_int64),
                 ("B", C.c_void_p), ("ldb", C.c_int64), ("Y", C.c_void_p), ("ldy", C.c_int64), ("d_out", C.c_int32)]
 
 
@@ -170,6 +178,11 @@ def _declare(L):
         L.cwl_ladder_build.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
                                        C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_size_t, C.POINTER(C.c_int32), C.c_void_p]
+        L.cwl_apply_batch_workspace_bytes.restype = C.c_size_t
+        L.cwl_apply_batch_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.c_int32]
+        L.cwl_apply_batch.restype = C.c_int
+        L.cwl_apply_batch.argtypes = [C.POINTER(CBatchItem), C.c_int32, C.c_int32, C.c_int32, CChunkTable, C.c_void_p, C.c_int32,
+                                      C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         L.cwl_set_pair_budget.restype = C.c_int
         L.cwl_set_pair_budget.argtypes = [C.c_int32]
         L.cwl_prefetch_next.restype = C.c_int
@@ -476,6 +489,44 @@ def cwl_ladder_build(A: torch.Tensor, B: torch.Tensor, want_f32: bool = True,
         _p(out.get("A32")), _p(out.get("B32")), _p(out["sigma"]), _p(ws), ws.numel(), C.byref(sweeps), _stream_ptr(stream)))
     out["sweeps"] = int(sweeps.value)
     return out
+
+
+def cwl_apply_batch_workspace_bytes(T: int, d_ins: Sequence[int], d_outs: Sequence[int], R: int) -> int:
+    n = len(d_ins)
+    a = (C.c_int32 * n)(*[int(d) for d in d_ins])
+    b = (C.c_int32 * n)(*[int(d) for d in d_outs])
+    return int(lib().cwl_apply_batch_workspace_bytes(T, n, a, b, R))
+
+
+class BatchCall:
+    """A batch of independent projections with everything marshalled once: the item descriptors are built at
+    construction, so a call costs one foreign call (decode steps are short enough for marshalling to show)."""
+
+    def __init__(self, Xs: Sequence[torch.Tensor], Ws: Sequence[torch.Tensor], As: Optional[Sequence[torch.Tensor]],
+                 Bs: Optional[Sequence[torch.Tensor]], Ys: Sequence[torch.Tensor], workspace: Optional[torch.Tensor] = None):
+        n = len(Ws)
+        self.T = int(Xs[0].shape[0])
+        self.R = int(As[0].shape[1]) if As is not None else 0
+        self.items = (CBatchItem * n)()
+        for j in range(n):
+            X, W, Y = Xs[j], Ws[j], Ys[j]
+            assert X.dtype == torch.bfloat16 and W.dtype == torch.bfloat16 and X.shape[0] == self.T
+            A = As[j] if As is not None else None
+            B = Bs[j] if Bs is not None else None
+            self.items[j] = CBatchItem(_p(X), X.stride(0), X.shape[1], _p(W), W.stride(0), _p(A), A.stride(0) if A is not None else 0,
+                                       _p(B), B.stride(0) if B is not None else 0, _p(Y), Y.stride(0), W.shape[1])
+        self.n = n
+        self.keep = (list(Xs), list(Ws), list(As or []), list(Bs or []), list(Ys))
+        need = cwl_apply_batch_workspace_bytes(self.T, [int(x.shape[1]) for x in Xs], [int(w.shape[1]) for w in Ws], self.R)
+        self.workspace = workspace if workspace is not None else torch.empty(need, dtype=torch.uint8, device=Ws[0].device)
+        assert self.workspace.numel() >= need
+
+    def __call__(self, table: Optional["DeviceChunkTable"], window: int, gates: Optional[torch.Tensor] = None,
+                 status_word: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> None:
+        ct = table.c_struct() if table is not None else CChunkTable(None, None, None, None, None, None, 0)
+        _check("cwl_apply_batch", lib().cwl_apply_batch(self.items, self.n, self.T, self.R, ct, _p(gates), int(window),
+                                                        _p(self.workspace), self.workspace.numel(), _p(status_word),
+                                                        _stream_ptr(stream)))
 
 
 def cwl_set_pair_budget(pairs: int) -> None:

@@ -461,8 +461,7 @@ static_assert(SmemLayout::kTotal <= 227 * 1024, "shared memory budget");
 // tiles), kSplitK = true for plans that split every tile's K loop over several pairs (the epilogue hands partial
 // accumulators over).  A launch runs exactly one of the two epilogues, so neither carries the other's code.
 template <bool kSplitK>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ ApplyParams p) {
+__device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParams& p, const int pair) {
   using L = SmemLayout;
   constexpr uint32_t kTmemCols = kMaxTileW;
 
@@ -492,7 +491,6 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair (issues the MMAs)
-  const int pair = blockIdx.x >> 1;
   const Plan& pl = p.plan;
   const int n_stages = pl.stages;
   const uint32_t stage_bytes = kABytes + pl.boxes * kBoxBytes;
@@ -978,6 +976,36 @@ apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ Apply
   }
 }
 
+template <bool kSplitK>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+apply_kernel(const __grid_constant__ GroupMaps tm, const __grid_constant__ ApplyParams p) {
+  apply_body<kSplitK>(tm, p, (int)(blockIdx.x >> 1));
+}
+
+// Several independent projections in ONE launch (cwl_apply_batch): every projection has its own run of CTA pairs and
+// its own plan, operands, workspace and sync words, exactly as if it had been launched alone on that many pairs; a pair
+// looks up which projection it belongs to and does that projection's work.  The projections share nothing but the
+// launch, so their set-up and their drains overlap one another's main loops, and consecutive batch launches chain like
+// any other launch of the library.
+struct BatchArgs {
+  int n;
+  int first_pair[CWL_MAX_BATCH + 1];   // projection j owns pairs [first_pair[j], first_pair[j + 1])
+  int split[CWL_MAX_BATCH];            // its plan splits the K loop (which epilogue it runs)
+  GroupMaps maps[CWL_MAX_BATCH];
+  ApplyParams params[CWL_MAX_BATCH];
+};
+
+static_assert(sizeof(BatchArgs) <= 16 * 1024, "kernel parameters of the batch launch");
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+apply_batch_kernel(const __grid_constant__ BatchArgs a) {
+  const int gp = (int)(blockIdx.x >> 1);
+  int j = 0;
+  while (j + 1 < a.n && gp >= a.first_pair[j + 1]) ++j;
+  if (a.split[j]) apply_body<true>(a.maps[j], a.params[j], gp - a.first_pair[j]);
+  else apply_body<false>(a.maps[j], a.params[j], gp - a.first_pair[j]);
+}
+
 // ------------------------------------------------------------------------------- host: the plan
 // Cost model, in KB of operands a CTA stages per K block: (16 KB of rows + 8 KB per right-operand box), plus a
 // per-tile epilogue term.  (Measured with the loads or the MMAs taken out of the loop, a 512-wide tile is bound by
@@ -1361,35 +1389,41 @@ cwl_status check_group(const void* X, int64_t ldx, const cwl_projection* proj, i
 }
 
 // Plans, carves the workspace, builds the tensor maps and launches one fused kernel for a group of projections.
-cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* proj, int n_proj, int32_t T,
-                            int32_t d_in, int32_t R, cwl_chunk_table table, int32_t window, void* workspace,
-                            size_t workspace_bytes, int32_t* status_word, void* stream_, bool allow_split_k,
-                            size_t scratch_limit, const cwl_row_gate* row_gates = nullptr,
-                            int32_t window_mode = CWL_WINDOW_CAUSAL) {
-  // the calling thread's one-shot prefetch hint belongs to this call, whatever becomes of it
-  const NextPrefetch hint = t_next_prefetch;
-  t_next_prefetch = {nullptr, 0};
+// Everything one launch (or one projection of a batch launch) needs: plan, carved workspace, tensor maps, parameters.
+struct Prepared {
+  GroupMaps maps;
+  ApplyParams p;
+  ApplyWorkspace ws;
+  bool uses_sync;          // has sync words (adapter or split K)
+};
+
+// Checks the arguments, plans for `pairs` CTA pairs, carves the workspace and builds tensor maps and kernel parameters.
+// *launch comes back false when there is nothing to do (T == 0).
+cwl_status prepare_group(const void* X, int64_t ldx, const cwl_projection* proj, int n_proj, int32_t T, int32_t d_in,
+                         int32_t R, cwl_chunk_table table, int32_t window, void* workspace, size_t workspace_bytes,
+                         int32_t* status_word, int pairs, bool allow_split_k, size_t scratch_limit,
+                         const cwl_row_gate* row_gates, int32_t window_mode, Prepared& out, bool* launch) {
+  *launch = false;
   bool adapter = false;
   const cwl_status chk = check_group(X, ldx, proj, n_proj, T, d_in, R, table, row_gates, window, adapter);
   if (chk != CWL_OK) return chk;
   if (T == 0) return CWL_OK;
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   const int Reff = adapter ? R : 0;
   int d_out[CWL_MAX_GROUP];
   for (int j = 0; j < n_proj; ++j) d_out[j] = proj[j].d_out;
 
   ApplyWorkspace ws{nullptr, nullptr, nullptr, nullptr, 0};
-  Plan pl = make_plan(T, d_in, n_proj, d_out, Reff, pairs_now(), allow_split_k, scratch_limit);
+  Plan pl = make_plan(T, d_in, n_proj, d_out, Reff, pairs, allow_split_k, scratch_limit);
   const size_t need = carve_apply(ws, static_cast<char*>(workspace), pl, T, Reff);
   const bool have_ws = workspace != nullptr && workspace_bytes >= need && (reinterpret_cast<uintptr_t>(workspace) & 255u) == 0;
   if (!have_ws && !adapter && pl.split_k > 1) {
     // the plain projection needs scratch only when its K loop is split; without a workspace it runs unsplit
-    pl = make_plan(T, d_in, n_proj, d_out, Reff, pairs_now(), false, scratch_limit);
+    pl = make_plan(T, d_in, n_proj, d_out, Reff, pairs, false, scratch_limit);
   } else if (!have_ws && (adapter || pl.split_k > 1)) {
     return CWL_ERR_WORKSPACE;
   }
 
-  GroupMaps maps;
+  GroupMaps& maps = out.maps;
   memset(&maps, 0, sizeof(maps));
   if (!make_map(&maps.x, X, (uint64_t)d_in, (uint64_t)T, (uint64_t)ldx, BK, BM)) return CWL_ERR_CUDA;
   maps.h = maps.x;                                  // never dereferenced when R == 0
@@ -1404,7 +1438,8 @@ cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* pr
     }
   }
 
-  ApplyParams p{};
+  ApplyParams& p = out.p;
+  p = ApplyParams{};
   p.T = T; p.d_in = d_in; p.R = Reff; p.RT = n_proj * Reff;
   p.window = window; p.window_mode = window_mode;
   for (int j = 0; j < n_proj; ++j) { p.Y[j] = static_cast<__nv_bfloat16*>(proj[j].Y); p.ldy[j] = proj[j].ldy; }
@@ -1417,44 +1452,90 @@ cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* pr
   p.wait_limit_ns = kWaitLimitNs; p.withhold_publish = 0;
 #endif
   p.plan = pl;
-  p.pf_ptr = hint.ptr; p.pf_bytes = hint.bytes;
-
   // Every launch tags its sync words with a fresh epoch, so words left by earlier launches (or never written) read as
   // zero and the workspace needs no clearing: a memset between two kernels costs ~5 us of idle GPU.  Only a launch
   // that is being captured into a CUDA graph is replayed with the same epoch; it records a clearing node instead.
   p.epoch = next_epoch();
-  cudaStreamCaptureStatus capture = cudaStreamCaptureStatusNone;
-  CWL_CUDA_TRY(cudaStreamIsCapturing(stream, &capture));
-  if (adapter || pl.split_k > 1) {
-    // (the entry point on the library's own scratch array, the one caller with a scratch limit, clears on every call)
-    if (capture != cudaStreamCaptureStatusNone || scratch_limit > 0)
-      CWL_CUDA_TRY(cudaMemsetAsync(ws.sync, 0, ws.sync_bytes, stream));
-  }
+  out.ws = ws;
+  out.uses_sync = adapter || pl.split_k > 1;
+  *launch = true;
+  return CWL_OK;
+}
 
-  static bool configured[64] = {};  // per device; benign race: the attribute call is idempotent
+cwl_status configure_kernels() {
+  static bool configured[64] = {};  // per device; benign race: the attribute calls are idempotent
   int dev = 0;
   CWL_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64 || !configured[dev]) {
     CWL_CUDA_TRY(cudaFuncSetAttribute(apply_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout::kTotal));
     CWL_CUDA_TRY(cudaFuncSetAttribute(apply_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout::kTotal));
+    CWL_CUDA_TRY(cudaFuncSetAttribute(apply_batch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout::kTotal));
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
-  // The kernel-to-kernel gap of a stream (~5 us for this cluster launch) is hidden by letting the launch overlap
-  // the tail of whatever kernel precedes it in the stream; the kernel itself waits for that kernel to complete
-  // before it touches global memory.  Captured launches keep the plain stream order.
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(2 * pl.pairs, 1, 1);
+  return CWL_OK;
+}
+
+// The kernel-to-kernel gap of a stream (~5 us for this cluster launch) is hidden by letting the launch overlap
+// the tail of whatever kernel precedes it in the stream; the kernel itself waits for that kernel to complete
+// before it touches global memory.  Captured launches keep the plain stream order.
+void launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute& attr, int pairs, cudaStream_t stream, bool capturing) {
+  cfg = cudaLaunchConfig_t{};
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = SmemLayout::kTotal;
   cfg.stream = stream;
-  cudaLaunchAttribute attr;
   attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
-  cfg.numAttrs = capture == cudaStreamCaptureStatusNone ? 1 : 0;
-  if (pl.split_k > 1) CWL_CUDA_TRY(cudaLaunchKernelEx(&cfg, apply_kernel<true>, maps, p));
-  else CWL_CUDA_TRY(cudaLaunchKernelEx(&cfg, apply_kernel<false>, maps, p));
+  cfg.numAttrs = capturing ? 0 : 1;
+}
+
+// Plans, carves the workspace, builds the tensor maps and launches one fused kernel for a group of projections.
+cwl_status apply_group_impl(const void* X, int64_t ldx, const cwl_projection* proj, int n_proj, int32_t T,
+                            int32_t d_in, int32_t R, cwl_chunk_table table, int32_t window, void* workspace,
+                            size_t workspace_bytes, int32_t* status_word, void* stream_, bool allow_split_k,
+                            size_t scratch_limit, const cwl_row_gate* row_gates = nullptr,
+                            int32_t window_mode = CWL_WINDOW_CAUSAL) {
+  // the calling thread's one-shot prefetch hint belongs to this call, whatever becomes of it
+  const NextPrefetch hint = t_next_prefetch;
+  t_next_prefetch = {nullptr, 0};
+  Prepared pr;
+  bool launch = false;
+  const cwl_status st = prepare_group(X, ldx, proj, n_proj, T, d_in, R, table, window, workspace, workspace_bytes,
+                                      status_word, pairs_now(), allow_split_k, scratch_limit, row_gates, window_mode, pr,
+                                      &launch);
+  if (st != CWL_OK || !launch) return st;
+  pr.p.pf_ptr = hint.ptr; pr.p.pf_bytes = hint.bytes;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  cudaStreamCaptureStatus capture = cudaStreamCaptureStatusNone;
+  CWL_CUDA_TRY(cudaStreamIsCapturing(stream, &capture));
+  const bool capturing = capture != cudaStreamCaptureStatusNone;
+  // (the entry point on the library's own scratch array, the one caller with a scratch limit, clears on every call)
+  if (pr.uses_sync && (capturing || scratch_limit > 0))
+    CWL_CUDA_TRY(cudaMemsetAsync(pr.ws.sync, 0, pr.ws.sync_bytes, stream));
+  const cwl_status cs = configure_kernels();
+  if (cs != CWL_OK) return cs;
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr;
+  launch_config(cfg, attr, pr.p.plan.pairs, stream, capturing);
+  if (pr.p.plan.split_k > 1) CWL_CUDA_TRY(cudaLaunchKernelEx(&cfg, apply_kernel<true>, pr.maps, pr.p));
+  else CWL_CUDA_TRY(cudaLaunchKernelEx(&cfg, apply_kernel<false>, pr.maps, pr.p));
   return CWL_OK;
+}
+
+// How the resident pairs are shared among the projections of a batch: in proportion to the bytes of their weights,
+// at least one pair each.
+void batch_shares(int n, const int* d_in, const int* d_out, int pairs, int* share) {
+  double total = 0;
+  for (int j = 0; j < n; ++j) total += (double)d_in[j] * d_out[j];
+  int given = 0;
+  for (int j = 0; j < n; ++j) {
+    share[j] = (int)((double)d_in[j] * d_out[j] / total * pairs);
+    if (share[j] < 1) share[j] = 1;
+    given += share[j];
+  }
+  for (int j = 0; given < pairs; j = (j + 1) % n) { ++share[j]; ++given; }
+  for (int j = 0; given > pairs; j = (j + 1) % n) if (share[j] > 1) { --share[j]; --given; }
 }
 
 cwl_status apply_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, const void* A, int64_t lda,
@@ -1571,6 +1652,77 @@ extern "C" cwl_status cwl_apply_rows(const void* X, int64_t ldx, const void* W, 
   memset(&none, 0, sizeof(none));
   return cwl::apply_group_impl(X, ldx, &q, 1, T, d_in, R, none, 0, workspace, workspace_bytes, status_word, stream,
                                true, 0, gates);
+}
+
+extern "C" size_t cwl_apply_batch_workspace_bytes(int32_t T, int32_t n, const int32_t* d_in, const int32_t* d_out,
+                                                  int32_t R) {
+  if (T <= 0 || n < 1 || n > CWL_MAX_BATCH || d_in == nullptr || d_out == nullptr || R < 0) return 256;
+  int share[CWL_MAX_BATCH];
+  int di[CWL_MAX_BATCH], dn[CWL_MAX_BATCH];
+  for (int j = 0; j < n; ++j) { if (d_in[j] < 1 || d_out[j] < 1) return 256; di[j] = d_in[j]; dn[j] = d_out[j]; }
+  cwl::batch_shares(n, di, dn, cwl::pairs_now() < n ? n : cwl::pairs_now(), share);
+  size_t total = 0;
+  for (int j = 0; j < n; ++j) {
+    cwl::ApplyWorkspace w;
+    const cwl::Plan pl = cwl::make_plan(T, di[j], 1, &dn[j], R, share[j], true);
+    total += cwl::carve_apply(w, nullptr, pl, T, R);
+  }
+  return total;
+}
+
+extern "C" cwl_status cwl_apply_batch(const cwl_batch_item* items, int32_t n, int32_t T, int32_t R,
+                                      cwl_chunk_table table, const cwl_row_gate* gates, int32_t window,
+                                      void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream_) {
+  using namespace cwl;
+  t_next_prefetch = {nullptr, 0};                     // a pending hint is consumed, unused
+  if (items == nullptr || n < 1 || n > CWL_MAX_BATCH) return CWL_ERR_INVALID_ARG;
+  const int pairs = pairs_now();
+  if (pairs < n) return CWL_ERR_UNSUPPORTED;
+  int di[CWL_MAX_BATCH], dn[CWL_MAX_BATCH], share[CWL_MAX_BATCH];
+  for (int j = 0; j < n; ++j) {
+    if (items[j].d_in < 1 || items[j].d_out < 1) return CWL_ERR_INVALID_ARG;
+    di[j] = items[j].d_in; dn[j] = items[j].d_out;
+  }
+  batch_shares(n, di, dn, pairs, share);
+
+  static thread_local BatchArgs args;                 // 10 KB: not on the stack of every caller
+  args.n = 0;
+  args.first_pair[0] = 0;
+  char* ws = static_cast<char*>(workspace);
+  size_t left = workspace_bytes;
+  Prepared pr;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  cudaStreamCaptureStatus capture = cudaStreamCaptureStatusNone;
+  CWL_CUDA_TRY(cudaStreamIsCapturing(stream, &capture));
+  const bool capturing = capture != cudaStreamCaptureStatusNone;
+  for (int j = 0; j < n; ++j) {
+    const cwl_batch_item& it = items[j];
+    const bool adapter = it.A != nullptr && it.B != nullptr && R > 0;
+    cwl_projection q;
+    q.W = it.W; q.ldw = it.ldw; q.A = adapter ? it.A : nullptr; q.lda = it.lda; q.B = adapter ? it.B : nullptr; q.ldb = it.ldb;
+    q.Y = it.Y; q.ldy = it.ldy; q.d_out = it.d_out;
+    bool launch = false;
+    const cwl_status st = prepare_group(it.X, it.ldx, &q, 1, T, it.d_in, R, table, window, ws, left, status_word, share[j],
+                                        true, 0, gates, CWL_WINDOW_CAUSAL, pr, &launch);
+    if (st != CWL_OK) return st;
+    if (!launch) return CWL_OK;                       // T == 0
+    ApplyWorkspace unused;
+    const size_t used = carve_apply(unused, nullptr, pr.p.plan, T, pr.p.R);
+    if (ws != nullptr) { ws += used; left = left >= used ? left - used : 0; }
+    if (pr.uses_sync && capturing) CWL_CUDA_TRY(cudaMemsetAsync(pr.ws.sync, 0, pr.ws.sync_bytes, stream));
+    const int k = args.n++;
+    args.maps[k] = pr.maps;
+    args.params[k] = pr.p;
+    args.split[k] = pr.p.plan.split_k > 1 ? 1 : 0;
+    args.first_pair[k + 1] = args.first_pair[k] + pr.p.plan.pairs;
+  }
+  const cwl_status cs = configure_kernels();
+  if (cs != CWL_OK) return cs;
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr;
+  launch_config(cfg, attr, args.first_pair[args.n], stream, capturing);
+  CWL_CUDA_TRY(cudaLaunchKernelEx(&cfg, apply_batch_kernel, args));
+  return CWL_OK;
 }
 
 // ------------------------------------------------------------------------------ no-allocation variant

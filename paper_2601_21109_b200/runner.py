@@ -37,7 +37,7 @@ class HotPath:
 
     def __init__(self, w: Workload, device: str = "cuda", keep_host: bool = False, n_layers: int = 1,
                  grouped: bool = True, streaming: bool = False, share_weights: Optional["HotPath"] = None,
-                 prefetch_bytes: int = 0, concurrent: bool = True):
+                 prefetch_bytes: int = 0, concurrent: bool = True, decode_mode: Optional[str] = None):
         self.grouped = grouped
         self.prefetch_bytes = int(prefetch_bytes)    # decode: bytes of the next call's weights hinted to each call (0 = none)
         # decode with the token-by-token scheduler: every step the cached per-sequence state advances by one
@@ -88,7 +88,24 @@ class HotPath:
         # launch setting up and draining.  They are issued side by side on `lanes` streams, each call planned for its
         # share of the CTA pairs (cwl_set_pair_budget), so that one call's set-up and drain overlap the other's main
         # loop.  Every lane has a workspace of its own.
-        self.lanes = 2 if (concurrent and w.T < self.GROUP_MIN_T and len(w.projections) >= 2) else 1
+        # decode_mode: "batch" = the step's projections as ONE launch (cwl_apply_batch: the CTA pairs are shared out among
+        # them); "lanes" = side by side on two streams; "serial" = one after the other, each on the whole GPU.
+        decode_sized = w.T < self.GROUP_MIN_T and len(w.projections) >= 2
+        if decode_mode is None:
+            decode_mode = "batch" if concurrent else "serial"
+        self.decode_mode = decode_mode if decode_sized else "serial"
+        self.batch_calls = None
+        if self.decode_mode == "batch":
+            n = cwl.MAX_BATCH
+            self.batch_calls, self.batch_calls_dense = [], []
+            for projs in self.layers:
+                groups = [projs[i:i + n] for i in range(0, len(projs), n)]
+                self.batch_calls.append([cwl.BatchCall([self.X[p.d_in] for p in g], [p.W for p in g], [p.A for p in g],
+                                                       [p.B for p in g], [p.Y for p in g]) for g in groups])
+                self.batch_calls_dense.append([cwl.BatchCall([self.X[p.d_in] for p in g], [p.W for p in g], None, None,
+                                                             [p.Y for p in g], workspace=c.workspace)
+                                               for g, c in zip(groups, self.batch_calls[-1])])
+        self.lanes = 2 if self.decode_mode == "lanes" else 1
         if self.lanes > 1:
             self.lane_budget = [self.RESIDENT_PAIRS // self.lanes] * self.lanes
             self.lane_streams = [torch.cuda.Stream(device=device) for _ in range(self.lanes)]
@@ -174,6 +191,11 @@ class HotPath:
         can then follow one another without draining the GPU in between."""
         rows = self.streaming and table is None and not dense
         tab = table if table is not None else self.table
+        if self.batch_calls is not None:
+            for call in (self.batch_calls_dense if dense else self.batch_calls)[layer]:
+                call(None if (dense or rows) else tab, self.policy.window,
+                     gates=self.stream_state.gates if rows else None, status_word=self.status)
+            return
         if self.lanes > 1:
             # fork: the lanes start where the current stream stands; join: it continues once every lane is done
             if fork:
@@ -181,17 +203,19 @@ class HotPath:
                 self.fork_event.record(main)
                 for st in self.lane_streams:
                     st.wait_event(self.fork_event)
-            for i, p in enumerate(self.layers[layer]):
-                j = i % self.lanes
-                cwl.cwl_set_pair_budget(self.lane_budget[j])
-                if rows:
-                    cwl.cwl_apply_rows(self.X[p.d_in], p.W, p.A, p.B, self.stream_state.gates, Y=p.Y,
-                                       workspace=self.lane_ws[j], status_word=self.status, stream=self.lane_streams[j])
-                else:
-                    cwl.cwl_apply(self.X[p.d_in], p.W, None if dense else p.A, None if dense else p.B, tab,
-                                  self.policy.window, Y=p.Y, workspace=self.lane_ws[j], status_word=self.status,
-                                  stream=self.lane_streams[j])
-            cwl.cwl_set_pair_budget(0)
+            try:
+                for i, p in enumerate(self.layers[layer]):
+                    j = i % self.lanes
+                    cwl.cwl_set_pair_budget(self.lane_budget[j])
+                    if rows:
+                        cwl.cwl_apply_rows(self.X[p.d_in], p.W, p.A, p.B, self.stream_state.gates, Y=p.Y,
+                                           workspace=self.lane_ws[j], status_word=self.status, stream=self.lane_streams[j])
+                    else:
+                        cwl.cwl_apply(self.X[p.d_in], p.W, None if dense else p.A, None if dense else p.B, tab,
+                                      self.policy.window, Y=p.Y, workspace=self.lane_ws[j], status_word=self.status,
+                                      stream=self.lane_streams[j])
+            finally:
+                cwl.cwl_set_pair_budget(0)          # later calls of this thread plan for the whole GPU again
             if join:
                 self.join_lanes()
             return
@@ -242,7 +266,7 @@ class HotPath:
 
     def launches_per_step(self, layers: Optional[int] = None) -> int:
         """Kernel launches of one step through `layers` weight sets (default: the whole stack)."""
-        n = self.LAUNCHES_APPLY * len(self.launch_groups())
+        n = self.LAUNCHES_APPLY * (len(self.batch_calls[0]) if self.batch_calls is not None else len(self.launch_groups()))
         if self.logits is not None:
             n += self.LAUNCHES_SCORE
         if not self.fixed_table:
