@@ -57,7 +57,7 @@ def load_peaks():
 
 # Revision tag of the dominant kernel the ncu counters under profiles/ were taken on.  Bump it whenever
 # cwl_apply's kernel changes: a traffic figure taken on another revision is reported as null.
-APPLY_KERNEL_REVISION = "pairs-256x512-grouped-r8"
+APPLY_KERNEL_REVISION = "pairs-256x512-grouped-r9"
 
 
 def load_traffic(key: str):
@@ -422,21 +422,39 @@ def measure(name: str, args, steps: int, warmup: int, world: int, rank: int, loc
         torch.cuda.synchronize()
         apply_ms = sum(x.elapsed_time(y) for x, y in ev) / n2
 
-    # ---- decode with a fixed table: the same steps with the lanes left running (no join between steps; each lane keeps
-    # its order and the region ends with a join).  The steps of this workload do not depend on one another, so this is a
-    # legal schedule; the headline figure above keeps the join after every step.
+    # ---- decode: the same steps under the other schedules (the step's projections side by side on two streams; one after
+    # the other on the whole GPU), and, with a fixed table, with the two-stream lanes left running (no join between steps;
+    # each lane keeps its order and the region ends with a join: the steps of this workload do not depend on one another,
+    # so this is a legal schedule; every other figure keeps step i+1 behind step i).
     free_ms = None
-    if decode and not streaming and hp.lanes > 1 and not args.lean:
-        n3 = max(steps, int(math.ceil(0.5e3 / max(ms_per_step, 1e-3))))
-        x, y = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        x.record(stream)
-        for i in range(n3):
-            hp.apply_step(layer=i % n_layers, join=False, fork=(i == 0))
-        hp.join_lanes()
-        y.record(stream)
-        torch.cuda.synchronize()
-        free_ms = x.elapsed_time(y) / n3
+    other_modes = {}
+    if decode and not args.lean:
+        n3 = max(steps, int(math.ceil(1.0e3 / max(ms_per_step, 1e-3))))
+        for mode in ("batch", "lanes", "serial"):
+            if mode == hp.decode_mode:
+                continue
+            alt = HotPath(w, n_layers=n_layers, grouped=not args.no_group, streaming=streaming, share_weights=hp, decode_mode=mode)
+            for i in range(10):
+                alt.step(layer=i % n_layers)
+            x, y = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            x.record(stream)
+            for i in range(n3):
+                alt.step(layer=i % n_layers)
+            y.record(stream)
+            torch.cuda.synchronize()
+            other_modes[mode] = {"ms_per_step": x.elapsed_time(y) / n3, "steps": n3}
+            if mode == "lanes" and not streaming:
+                x.record(stream)
+                for i in range(n3):
+                    alt.apply_step(layer=i % n_layers, join=False, fork=(i == 0))
+                alt.join_lanes()
+                y.record(stream)
+                torch.cuda.synchronize()
+                free_ms = x.elapsed_time(y) / n3
+            if int(alt.status.item()) != 0:
+                raise SystemExit(f"device status word {int(alt.status.item()):#x}")
+            del alt
 
     # ---- comparison runs through the same kernels: static full-rank LoRA and the dense floor ---
     static_ms = dense_ms = chunk_only_ms = None
@@ -539,7 +557,7 @@ def measure(name: str, args, steps: int, warmup: int, world: int, rank: int, loc
            "n_chunks": int(table["n_chunks"]) if table is not None else None,
            "tflops": f_alg * n_steps * world / (ms_total * 1e-3) / 1e12,
            "apply_ms_per_step": apply_ms, "apply_only_loop_ms": chunk_only_ms, "decode_mode": hp.decode_mode if decode else None,
-           "free_running_lanes_ms_per_step": free_ms,
+           "other_decode_modes": other_modes or None, "free_running_lanes_ms_per_step": free_ms,
            "static_lora_apply_ms": static_ms, "dense_floor_apply_ms": dense_ms,
            "clocks": clocks, "gpu_launches": hp.launches_per_step(stack) * n_steps, "roofline": roof}
     if e2e is not None:

@@ -37,7 +37,7 @@ def test_matches_the_oracle_and_stays_inside_its_outputs(T, shapes, R):
     cuts = list(range(29, T, 41))
     n = len(cuts) + 1
     ranks = ([R, R // 2, R // 4] * n)[:n]
-    tab = simple_table(T, cuts, ranks, [32.0 / r for r in ranks], flags=[1] + [0] * (n - 1))
+    tab = simple_table(T, cuts, ranks, [float(R) / r for r in ranks], flags=[1] + [0] * (n - 1))   # scale = alpha / rank, alpha = R
     bufs = [guarded(T, d_out) for _, d_out in shapes]
     call = cwl.BatchCall([d["X"] for d in dev], [d["W"] for d in dev], [d["A"] for d in dev], [d["B"] for d in dev],
                          [y for _, y in bufs])
