@@ -320,6 +320,14 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------- our arm
+_T0 = time.time()
+
+
+def progress(what: str):
+    """Phase marks on stderr (stdout carries the one JSON line only)."""
+    print(f"[bench +{time.time() - _T0:6.1f}s] {what}", file=sys.stderr, flush=True)
+
+
 def measure(name: str, args, steps: int, warmup: int, world: int, rank: int, local_rank: int, full: bool):
     """Builds one workload on the device, times it, and returns (result dict, workload)."""
     import torch
@@ -328,9 +336,11 @@ def measure(name: str, args, steps: int, warmup: int, world: int, rank: int, loc
     from paper_2601_21109_b200 import workloads as wl
     from paper_2601_21109_b200.runner import HotPath
 
+    progress(f"{name}: generating the workload")
     w = make_workload(name)
     n_layers = layers_of(name, args)
     stack = n_layers if name == "cfg5" else 1           # layers one step runs through
+    progress(f"{name}: device buffers, plans")
     decode = name in ("cfg4", "cfg4_stream")
     streaming = name == "cfg4_stream"
     hp = HotPath(w, n_layers=n_layers, grouped=not args.no_group, streaming=streaming, prefetch_bytes=int(args.prefetch_mb * 1e6),
@@ -365,6 +375,7 @@ def measure(name: str, args, steps: int, warmup: int, world: int, rank: int, loc
     f_alg, f_exe = f_alg * stack, f_exe * stack
 
     # ---- device-resident timing: blocks of `steps` steps, no event inside a block ---------------
+    progress(f"{name}: warm-up and timed region")
     for i in range(warmup):
         run_step(i)
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -401,6 +412,7 @@ def measure(name: str, args, steps: int, warmup: int, world: int, rank: int, loc
     value = replicas.job_throughput(hp.T, n_steps, world, ms_total)
     ms_per_step = ms_total / n_steps
 
+    progress(f"{name}: apply launches alone, comparison runs")
     # ---- the apply launches alone, inside whole steps (second pass: the headline span above has no inner event) ----
     if decode and not streaming:
         apply_ms = ms_per_step                  # the step IS its apply launches
@@ -483,6 +495,7 @@ def measure(name: str, args, steps: int, warmup: int, world: int, rank: int, loc
     # ---- end to end: pinned host inputs in, results out, every step ----------------------------
     e2e = None
     if full and not args.lean:
+        progress(f"{name}: end to end with host buffers")
         from paper_2601_21109_b200.runner import HostPipeline
         pipe = HostPipeline(w, n_layers=n_layers, grouped=not args.no_group, first=hp, streaming=streaming)
         e2e_steps = max(4, min(steps, 20))
@@ -601,6 +614,7 @@ def run_ours(args):
     if args.lean or world > 1:
         cpu = {}
     else:
+        progress("oracle on the host cores")
         n_rows, _ = rows_for_budget(w, 25.0)         # about 10-20 s of CPU work
         cpu_val, cpu_info = oracle_sample(w, n_rows=n_rows)
         if stack > 1:
@@ -623,6 +637,7 @@ def run_ours(args):
     }
     if configs:
         line["configs"] = configs
+    progress("done")
     print(json.dumps(line))
     replicas.finish(world)
 
