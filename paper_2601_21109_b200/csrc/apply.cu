@@ -71,7 +71,7 @@ constexpr int kOutBufBytes = 4096;  // per epilogue warp: 32 rows x 64 bf16 colu
 constexpr int kThreads = 320;       // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: epilogue
 constexpr int kEpiThreads = 256;
 constexpr int kEpiWarps = 8;
-constexpr int kGroupM = 8;          // pair rows (256 tokens each) per raster group: their X rows stay L2-resident
+constexpr int kGroupM = 16;         // pair rows (256 tokens each) per raster group: a wave of tiles shares them (see raster())
 constexpr int kPairsPlanned = 74;   // most CTA pairs ever launched (148 SMs); plans never use more
 constexpr int kMaxSplits = 16;      // split factor of the shrink along d_in
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -173,6 +173,30 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
   asm volatile(
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(map), "r"(leader_bar), "r"(x), "r"(y) : "memory");
+}
+// The same with an L2 eviction policy for the lines it brings in.
+__device__ __forceinline__ void tma_load_2d_pair_hint(uint32_t dst, const CUtensorMap* map, uint32_t leader_bar, int x, int y,
+                                                      uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(map), "r"(leader_bar), "r"(x), "r"(y), "l"(policy) : "memory");
+}
+// L2 eviction policies: rows of X are read again by every column tile of their raster group (keep them), rows of Y are
+// written once and not read by this launch (let them go first).  W gets no hint: the pairs that share a column slab read it
+// within a short time of one another, and marking it for early eviction was measured to double its DRAM reads.
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void st_global_v4_hint(void* ptr, uint4 v, uint64_t policy) {
+  asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1, %2, %3, %4}, %5;"
+               ::"l"(ptr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "l"(policy) : "memory");
 }
 // contiguous global -> shared copy (16-byte aligned, a multiple of 16 bytes) counted on an mbarrier of this CTA
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -322,7 +346,8 @@ struct Item {
 };
 
 // Rastered tile index -> (pair row, column tile): groups of kGroupM pair rows, pair row fastest inside a
-// group, so that a group's X rows and the W column slabs stay in L2.
+// group.  The 74 tiles in flight then cover 16 pair rows x 4-5 column tiles, close to the smallest set of X rows and
+// W slabs 74 tiles can touch (about 50 MB at d_in = 4096), and the next 74 need the same X rows again.
 __device__ __forceinline__ void raster(int tile, int n_m_pairs, int n_cols, int& m_pair, int& c) {
   const int per_group = kGroupM * n_cols;
   const int group = tile / per_group, within = tile - group * per_group;
@@ -542,6 +567,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
       uint32_t s = 0, ph = 0;   // ring slot and phase parity of it_cnt, kept incrementally (no division per step)
       const uint32_t leader_full0 = mapa_shared(full_bar(0), 0);   // full_bar(0) in the leader's shared memory
       bool ok = true;
+      const uint64_t keep_x = policy_evict_last();
       Item item;
       for (int i = 0; ok && get_item(i, pair, sh_begin, p, item); ++i) {
         const bool shrink = item.kind == ITEM_SHRINK;
@@ -577,7 +603,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
           if (lane == 0) {
             if (rank == 0) mbar_expect_tx(full_bar(s), tx_pair);
             if (phase1) tma_load_2d_pair(sa, &tm.h, leader_full, item.proj * p.R + k, m_tile * BM);
-            else tma_load_2d_pair(sa, &tm.x, leader_full, k, m_tile * BM);
+            else tma_load_2d_pair_hint(sa, &tm.x, leader_full, k, m_tile * BM, keep_x);
           } else if (has_box) {
             tma_load_2d_pair(sb + bi * kBoxBytes, phase1 ? map1 : map0, leader_full, box_x, k);
           }
@@ -735,7 +761,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
           for (int k = 0; k < 8; ++k) {
             const int r = (lane >> 3) + 4 * k;       // lanes 8j..8j+7 take the eight pieces of row r
             const uint4 q = ld_shared_v4(obuf + r * 128 + (((lane & 7) ^ (r & 7)) << 4));
-            if (row0 + r < p.T) *reinterpret_cast<uint4*>(out + (int64_t)(row0 + r) * ldy) = q;
+            if (row0 + r < p.T) st_global_v4_hint(out + (int64_t)(row0 + r) * ldy, q, policy_evict_first());
           }
         }
         const int rem = item.wt & 63;                // a last chunk of 16, 32 or 48 columns: plain 16-byte stores
