@@ -25,6 +25,22 @@ void cwl_debug_set(int64_t wait_limit_ns, int32_t withhold_publish);
  * Errors: INVALID_ARG, CUDA; a wait that runs out flags CWL_ERR_TIMEOUT in *status_word. */
 cwl_status cwl_probe_read(const void* ptr, size_t bytes, int32_t* status_word, void* stream);
 
+/* Device timeline of one CTA pair of the apply kernels (any cwl_apply* call made afterwards).  The leader CTA of
+ * pair `pair` (blockIdx.x / 2 of the launch; in a batch launch pairs are numbered through all projections) writes
+ * %globaltimer readings (ns, 32 ns granularity) into slots[0..1023]; every launch overwrites the slots, so read them
+ * after the launch of interest.  slots == NULL or pair < 0 switches tracing off.
+ *   slots  DEV, 1024 int64, zeroed by the caller.
+ *   [0] kernel entered   [1] the launch ahead in the stream has finished (griddepcontrol.wait returned)
+ *   [2] last accumulator committed by the MMA issuer   [5] epilogue saw the last accumulator
+ *   [3] epilogue left its item loop   [4] CTA barrier of the teardown passed
+ *   split-K hand-over: [6] partial sums stored  [7] all contributors arrived  [8] their sums copied in  [9] reduced and staged
+ *   shrink epilogue:   [11] partial sums stored and fenced  [12] arrival counted  [13] reduced (last arriver only)  [14] fenced
+ *   [15],[16] producer: wait for the H' flag begins / ends
+ *   K block i of the pair (running count over its items, i < 290): [100+i] loads issued, [400+i] operands landed
+ *   (MMA issuer's wait returned), [700+i] MMAs issued and committed.
+ * Errors: CUDA. */
+cwl_status cwl_trace_set(long long* slots, int32_t pair);
+
 #ifdef __cplusplus
 }
 #endif

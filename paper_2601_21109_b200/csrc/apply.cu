@@ -155,6 +155,20 @@ __device__ __forceinline__ unsigned long long global_timer() {
 __device__ __forceinline__ unsigned long long wait_limit(volatile int* abort_flag) {
   return *reinterpret_cast<volatile unsigned long long*>(abort_flag + 3);
 }
+#ifdef CWL_TEST_HOOKS
+// Test build only (cwl_trace_set): the leader CTA of one chosen pair writes %globaltimer readings of its producer, its
+// MMA issuer and its first epilogue thread into a caller-supplied array; the slots are listed in cwl_test_hooks.h.
+__device__ long long* g_trace = nullptr;
+__device__ int g_trace_pair = -1;
+#define CWL_TRACE_DECL const bool tr = g_trace != nullptr && (int)(blockIdx.x >> 1) == g_trace_pair && cluster_ctarank() == 0
+#define CWL_TRACE(i) do { if (tr) g_trace[(i)] = (long long)global_timer(); } while (0)
+#define CWL_TRACE_N(base, i) do { if (tr && (i) < 290u) g_trace[(base) + (i)] = (long long)global_timer(); } while (0)
+#else
+#define CWL_TRACE_DECL do {} while (0)
+#define CWL_TRACE(i) do {} while (0)
+#define CWL_TRACE_N(base, i) do {} while (0)
+#endif
+
 // Bounded wait.  Returns false when the limit ran out or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -556,7 +570,10 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
     const bool any = get_item(0, pair, sh_begin, p, warm);
     asm volatile("" ::"r"(warm.wt + warm.kb0 + warm.n_blk0 + warm.n0 + (any ? 1 : 0)));
   }
-  asm volatile("griddepcontrol.wait;" ::: "memory");   // nothing before this line reads or writes global memory
+  CWL_TRACE_DECL;
+  if (threadIdx.x == 32) CWL_TRACE(0);
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // nothing before this line reads or writes global memory (but a trace)
+  if (threadIdx.x == 32) CWL_TRACE(1);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -593,7 +610,9 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
           const bool phase1 = b >= item.n_blk0;
           if (phase1 && b == item.n_blk0) {
             // H' of this CTA's row tile must have been published by whoever finished its shrink
+            if (lane == 0) CWL_TRACE(15);
             if (lane == 0 && step_ok) step_ok = wait_word(p.flags + m_tile * pl.n_proj + item.proj, p.epoch, 1, abort_flag);
+            if (lane == 0) CWL_TRACE(16);
             fence_proxy_async();
           }
           if (!__all_sync(0xffffffffu, step_ok)) { ok = false; break; }
@@ -601,6 +620,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
           const uint32_t sa = base + s * stage_bytes, sb = sa + kABytes;
           const uint32_t leader_full = leader_full0 + 8u * s;      // this stage's barrier in the leader's shared memory
           if (lane == 0) {
+            CWL_TRACE_N(100, it_cnt);
             if (rank == 0) mbar_expect_tx(full_bar(s), tx_pair);
             if (phase1) tma_load_2d_pair(sa, &tm.h, leader_full, item.proj * p.R + k, m_tile * BM);
             else tma_load_2d_pair_hint(sa, &tm.x, leader_full, k, m_tile * BM, keep_x);
@@ -647,6 +667,9 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
       uint32_t s = 0, ph = 0;   // ring slot and phase parity, kept incrementally
       bool ok = true;
       Item item;
+#ifdef CWL_TEST_HOOKS
+      uint32_t blocks_done = 0;   // K blocks issued so far, over all items (trace slots)
+#endif
       // descriptors of ring slot 0; a slot is stage_bytes further on (the address field counts 16-byte units and the
       // whole ring lies below 256 KB, so adding to the 64-bit descriptor never carries out of the field)
       const uint64_t desc_a0 = make_smem_desc(base, 16, 1024);
@@ -668,6 +691,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
         const int tail1 = (p.R & (BK - 1)) != 0 ? (p.R & (BK - 1)) / UMMA_K : BK / UMMA_K;
         for (int b = 0; b < n_blk; ++b) {
           if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+          CWL_TRACE_N(400, blocks_done);
           tc_fence_after();
           int k_steps = BK / UMMA_K;
           if (b == item.n_blk0 - 1) k_steps = tail0;
@@ -692,10 +716,15 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
             }
           }
           umma_commit_pair(empty_bar(s));            // frees the stage in both CTAs once these MMAs have read it
+#ifdef CWL_TEST_HOOKS
+          CWL_TRACE_N(700, blocks_done);
+          ++blocks_done;
+#endif
           if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; da = desc_a0; db = desc_b0; }
           else { da += desc_slot; db += desc_slot; }
         }
         if (ok) umma_commit_pair(acc_full_bar);      // accumulator complete, both CTAs
+        CWL_TRACE(2);
       }
       if (!ok) {
         // give the MMAs still in flight a bounded time to retire before TMEM is released
@@ -718,6 +747,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
         gates[epi_tid] = row_gate((item.m_pair * 2 + (int)rank) * BM + epi_tid, p);
       }
       mbar_wait(acc_full_bar, local & 1u, abort_flag);    // a failure is recorded in abort_flag
+      if (threadIdx.x == 64) CWL_TRACE(5);
       // one thread decides for all 256 so that the barriers below are never split
       epilogue_barrier();
       if (epi_tid == 0) *epi_go = (*abort_flag == 0);
@@ -821,6 +851,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
           }
         }
         epilogue_barrier();                          // every thread's partial stores precede thread 0's release below
+        if (threadIdx.x == 64) CWL_TRACE(6);
         unsigned long long* counter = p.sk_counters + item.tile * 2 + rank;
         // The others' partial sums of this CTA's share are one contiguous run per contributor: where they fit the
         // (now idle) operand ring beside the staged rows, bulk copies bring them in at once instead of a chain of
@@ -832,6 +863,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
           __threadfence();                           // device-wide release of the CTA's partial (cumulative over the barrier)
           sync_arrive(counter, p.epoch);
           bool in = wait_word(counter, p.epoch, pl.split_k, abort_flag);
+          CWL_TRACE(7);
           if (in && landed) {
             fence_proxy_async();                     // the partials were written with ordinary stores
             mbar_expect_tx(fix_bar, (uint32_t)(pl.split_k - 1) * seg_bytes);
@@ -844,6 +876,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
             in = mbar_wait(fix_bar, 0, abort_flag);  // bounded; a failure is recorded in abort_flag
           }
           *epi_go = in ? 1 : 0;
+          CWL_TRACE(8);
         }
         epilogue_barrier();
         if (*epi_go == 0) break;
@@ -903,6 +936,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(leader_acc_empty);
         epilogue_barrier();
+        if (threadIdx.x == 64) CWL_TRACE(9);
         const int pieces = (c_hi - c_lo) >> 3;       // 16-byte pieces per row
         for (int idx = epi_tid; idx < BM * pieces; idx += kEpiThreads) {
           const int r = idx / pieces, pc = idx - r * pieces;
@@ -961,39 +995,64 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
         if (epi_tid == 0 && !p.withhold_publish) st_release(p.flags + sync_idx, p.epoch | 1ull);
         continue;
       }
+      if (threadIdx.x == 64) CWL_TRACE(11);
       if (epi_tid == 0) *epi_last = (sync_arrive(p.counters + sync_idx, p.epoch) == pl.shrink_splits - 1);
       epilogue_barrier();
+      if (threadIdx.x == 64) CWL_TRACE(12);
       if (*epi_last == 0) continue;
       // this CTA completed its projection's share of the row tile: sum the partials, gate, publish H'
       __threadfence();
       const int quads = p.R >> 2;                    // float4 groups per row of this projection
       const int64_t split_stride = (int64_t)2 * pl.n_m_pairs * p.RT * BM;
-      for (int idx = epi_tid; idx < BM * quads; idx += kEpiThreads) {
-        const int r = idx & (BM - 1), cg = idx >> 7, j0 = cg << 2;   // rank index
-        const int t = m_tile * BM + r;
-        if (t >= p.T) continue;
-        const RowGate gr = gates[r];
-        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-        const float* src = p.partial + (((int64_t)m_tile * (p.RT >> 2) + (hcol >> 2) + cg) * BM + r) * 4;
-#pragma unroll 4
-        for (int s = 0; s < pl.shrink_splits; ++s) {
-          const float4 x = __ldcg(reinterpret_cast<const float4*>(src + s * split_stride));
-          sum.x += x.x; sum.y += x.y; sum.z += x.z; sum.w += x.w;
+      // Every thread owns the groups idx = epi_tid + k * 256.  It takes them eight at a time and, split by split, loads
+      // the eight partial sums before it adds any of them: the loads of a batch are independent, so their latencies
+      // overlap (a loop that finished one group before it loaded the next one took one memory round trip per group).
+      constexpr int kBatch = 8;
+      for (int idx0 = epi_tid; idx0 < BM * quads; idx0 += kEpiThreads * kBatch) {
+        float4 sum[kBatch];
+        const float* src[kBatch];
+#pragma unroll
+        for (int g = 0; g < kBatch; ++g) {
+          const int idx = idx0 + g * kEpiThreads;
+          const int r = idx & (BM - 1), cg = idx >> 7;
+          const bool live = idx < BM * quads && m_tile * BM + r < p.T;
+          sum[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+          src[g] = live ? p.partial + (((int64_t)m_tile * (p.RT >> 2) + (hcol >> 2) + cg) * BM + r) * 4 : nullptr;
         }
-        uint2 o;
-        o.x = pack_bf16(sum.x * gate_at(gr, j0), sum.y * gate_at(gr, j0 + 1));
-        o.y = pack_bf16(sum.z * gate_at(gr, j0 + 2), sum.w * gate_at(gr, j0 + 3));
-        *reinterpret_cast<uint2*>(p.Hg + (int64_t)t * p.RT + hcol + j0) = o;
+#pragma unroll 2
+        for (int s = 0; s < pl.shrink_splits; ++s) {
+          float4 x[kBatch];
+#pragma unroll
+          for (int g = 0; g < kBatch; ++g)
+            x[g] = src[g] != nullptr ? __ldcg(reinterpret_cast<const float4*>(src[g] + s * split_stride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+          for (int g = 0; g < kBatch; ++g) { sum[g].x += x[g].x; sum[g].y += x[g].y; sum[g].z += x[g].z; sum[g].w += x[g].w; }
+        }
+#pragma unroll
+        for (int g = 0; g < kBatch; ++g) {
+          if (src[g] == nullptr) continue;
+          const int idx = idx0 + g * kEpiThreads;
+          const int r = idx & (BM - 1), cg = idx >> 7, j0 = cg << 2;   // rank index
+          const RowGate gr = gates[r];
+          uint2 o;
+          o.x = pack_bf16(sum[g].x * gate_at(gr, j0), sum[g].y * gate_at(gr, j0 + 1));
+          o.y = pack_bf16(sum[g].z * gate_at(gr, j0 + 2), sum[g].w * gate_at(gr, j0 + 3));
+          *reinterpret_cast<uint2*>(p.Hg + (int64_t)(m_tile * BM + r) * p.RT + hcol + j0) = o;
+        }
       }
+      if (threadIdx.x == 64) CWL_TRACE(13);
       __threadfence();
       epilogue_barrier();
+      if (threadIdx.x == 64) CWL_TRACE(14);
       if (epi_tid == 0 && !p.withhold_publish) st_release(p.flags + sync_idx, p.epoch | 1ull);
     }
   }
 
   // ---------------------------------------------------------------------- teardown
+  if (threadIdx.x == 64) CWL_TRACE(3);
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 64) CWL_TRACE(4);
   cluster_sync();   // neither CTA leaves (or frees TMEM) while the other may still signal it or write its TMEM
   if (threadIdx.x == 0 && *abort_flag) flag_status(p.status_word, CWL_ERR_TIMEOUT);
   if (warp == 1) {
@@ -1607,6 +1666,13 @@ extern "C" cwl_status cwl_prefetch_next(const void* ptr, size_t bytes) {
 extern "C" void cwl_debug_set(int64_t wait_limit_ns, int32_t withhold_publish) {
   cwl::g_wait_limit_ns.store(wait_limit_ns > 0 ? (unsigned long long)wait_limit_ns : cwl::kWaitLimitNs);
   cwl::g_withhold_publish.store(withhold_publish != 0 ? 1 : 0);
+}
+
+extern "C" cwl_status cwl_trace_set(long long* slots, int32_t pair) {
+  if (slots == nullptr) pair = -1;
+  if (cudaMemcpyToSymbol(cwl::g_trace, &slots, sizeof(slots)) != cudaSuccess) return CWL_ERR_CUDA;
+  if (cudaMemcpyToSymbol(cwl::g_trace_pair, &pair, sizeof(pair)) != cudaSuccess) return CWL_ERR_CUDA;
+  return CWL_OK;
 }
 #endif
 

@@ -35,9 +35,10 @@ def test_library_exports_every_declared_symbol(lib_path):
 
 def test_the_test_hook_exists_in_the_test_build_only(lib_path):
     from paper_2601_21109_b200 import build
-    assert not hasattr(ctypes.CDLL(lib_path), "cwl_debug_set")
     hooks = ctypes.CDLL(build.LIB_HOOKS)
-    assert hasattr(hooks, "cwl_debug_set")
+    for name in ("cwl_debug_set", "cwl_trace_set", "cwl_probe_read"):
+        assert not hasattr(ctypes.CDLL(lib_path), name), name
+        assert hasattr(hooks, name), name
     for name in declared_functions():                        # and everything else as well
         assert hasattr(hooks, name), name
 
