@@ -556,8 +556,13 @@ def measure(name: str, args, steps: int, warmup: int, world: int, rank: int, loc
                 "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
                 "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
                 "executed_tflops": f_exe / (apply_ms * 1e-3) / 1e12, "frac_of_nominal_2250": achieved / 2250.0}
-    roof["kernel"] = ("cwl::apply_kernel (one fused launch per projection or projection group: shrink, gate, base GEMM + "
-                      "expand); achieved = the step's algorithmic FLOPs or bytes over the event-timed span of its apply launches")
+    if decode and hp.decode_mode == "batch":
+        roof["kernel"] = ("cwl::apply_batch_kernel (the step's projections in one launch, each on its share of the CTA pairs: "
+                          "shrink, gate, base GEMM + expand); achieved = the step's algorithmic bytes over the event-timed "
+                          "span of its apply launches")
+    else:
+        roof["kernel"] = ("cwl::apply_kernel (one fused launch per projection or projection group: shrink, gate, base GEMM + "
+                          "expand); achieved = the step's algorithmic FLOPs or bytes over the event-timed span of its apply launches")
     roof["launch_ms"] = apply_ms
     roof["sm_mhz_median"] = clocks.get("sm_mhz") if clocks else None
     if clocks and clocks.get("sm_mhz"):
