@@ -341,7 +341,7 @@ cwl_status cwl_prefetch_next(const void* ptr, size_t bytes);
  *   split_k                 pairs sharing one tile's K loop (1 = none); k_blocks_per_split 64-deep blocks each
  *   shrink_splits           splits of d_in in the shrink; shrink_items = row_tiles * shrink_splits are handed
  *                           out over the pairs (shrink_items_assigned = their total, ..max_per_pair the most one pair gets)
- *   stages                  depth of the right-operand TMA ring;  model_cost: the planner's figure for the busiest pair
+ *   stages                  depth of the TMA ring;  model_cost: the planner's figure for the busiest pair
  * Errors: INVALID_ARG, UNSUPPORTED (same shape rules as cwl_apply). */
 typedef struct {
   int32_t pairs, row_tiles;

@@ -27,12 +27,10 @@
 //            an fp32 partial, and once all of a tile's partials are in, every contributor reduces its
 //            share of the tile's columns and writes Y.
 //
-// Roles per CTA: warp 0 = TMA producer of the right operand (cp.async.bulk.tensor, 128-byte swizzle, bytes
-// counted on the leader's mbarrier), warp 10 = TMA producer of the left operand, each with a ring of its own
-// (the left operand comes out of L2 and needs three or four slots; the rest of shared memory holds boxes of
-// the right operand, the bytes HBM has to deliver), warp 1 = tcgen05.mma issuer in the leader CTA only
-// (tcgen05.commit multicast frees the slots in both CTAs), warps 2..9 = epilogue (tcgen05.ld of the CTA's
-// own 128 accumulator rows; two warps per TMEM lane quadrant).  The left operand is K-major (rows of X / H'), the right
+// Roles per CTA: warp 0 = TMA producer (cp.async.bulk.tensor, 128-byte swizzle, bytes counted on the
+// leader's mbarrier), warp 1 = tcgen05.mma issuer in the leader CTA only (tcgen05.commit multicast
+// frees the stage in both CTAs), warps 2..9 = epilogue (tcgen05.ld of the CTA's own 128 accumulator
+// rows; two warps per TMEM lane quadrant).  The left operand is K-major (rows of X / H'), the right
 // operand is N-major (rows of W, A, B are contiguous in their output dimension), exactly as the
 // matrices sit in HBM.
 //
@@ -70,8 +68,7 @@ constexpr int kRingBytes = 192 * 1024;
 constexpr int kRingBytesSplit = 216 * 1024;
 constexpr int kOutBytesSplit = 8 * 1024;
 constexpr int kOutBufBytes = 4096;  // per epilogue warp: 32 rows x 64 bf16 columns staged for row-contiguous stores
-constexpr int kThreads = 352;       // warp 0: TMA (right operand), warp 1: MMA + TMEM owner, warps 2..9: epilogue, warp 10: TMA (left operand)
-constexpr int kLeftWarp = 10;
+constexpr int kThreads = 320;       // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: epilogue
 constexpr int kEpiThreads = 256;
 constexpr int kEpiWarps = 8;
 constexpr int kGroupM = 16;         // pair rows (256 tokens each) per raster group: a wave of tiles shares them (see raster())
@@ -95,8 +92,7 @@ struct Plan {
   int split_k, kb_per_ksplit; // split of the d_in blocks of every tile (1 = none); only when all items fit one wave
   int shrink_splits, kb_per_split;
   int boxes;                  // right-operand boxes per CTA per stage, at most
-  int stages;              // slots of the right-operand ring
-  int stages_x;            // slots of the left-operand ring
+  int stages;
   uint16_t sh_count[kPairsPlanned];  // shrink items per pair
   long long makespan;         // model cost of the busiest pair (diagnostic)
 };
@@ -492,7 +488,7 @@ __device__ __forceinline__ bool wait_word(const unsigned long long* word, unsign
 
 struct SmemLayout {
   static constexpr int kOutBytes = kEpiWarps * kOutBufBytes;   // also holds the row gates of a shrink finaliser
-  static constexpr int kBarBytes = (4 * kMaxStages + 3) * 8;
+  static constexpr int kBarBytes = (2 * kMaxStages + 3) * 8;
   static constexpr int kMiscBytes = 32;              // TMEM base, abort flag, epilogue broadcast words
   static constexpr int kTotal = kRingBytes + kOutBytes + kBarBytes + kMiscBytes + 1024;  // + alignment slack
 };
@@ -520,15 +516,11 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
   constexpr int kOut = kSplitK ? kOutBytesSplit : L::kOutBytes;
   const uint32_t out_bufs = base + kRing;           // per-warp staging buffers of the epilogue
   const uint32_t bars = out_bufs + kOut;
-  // two rings with barriers of their own: the right operand (W, A or B boxes: the bytes that come from HBM) and the
-  // left operand (128 rows of X or H', which come out of L2)
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
-  auto full_x = [&](int s) { return bars + 8u * (2 * kMaxStages + s); };
-  auto empty_x = [&](int s) { return bars + 8u * (3 * kMaxStages + s); };
-  const uint32_t acc_full_bar = bars + 8u * (4 * kMaxStages);
-  const uint32_t acc_empty_bar = bars + 8u * (4 * kMaxStages + 1);
-  const uint32_t fix_bar = bars + 8u * (4 * kMaxStages + 2);   // split-K: the others' partial sums have landed
+  const uint32_t acc_full_bar = bars + 8u * (2 * kMaxStages);
+  const uint32_t acc_empty_bar = bars + 8u * (2 * kMaxStages + 1);
+  const uint32_t fix_bar = bars + 8u * (2 * kMaxStages + 2);   // split-K: the others' partial sums have landed
   uint8_t* misc = base_ptr + kRing + kOut + L::kBarBytes;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
@@ -539,21 +531,14 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair (issues the MMAs)
   const Plan& pl = p.plan;
-  const int n_stages = pl.stages, n_stages_x = pl.stages_x;
-  const uint32_t stage_bytes = pl.boxes * kBoxBytes;            // one slot of the right-operand ring
-  const uint32_t ring_w = base + (uint32_t)n_stages_x * kABytes; // it follows the left-operand ring
-  // rings of equal depth turn together: one commit per K block then frees the slot of both (the left-operand producer waits
-  // on the right-operand ring's barrier)
-  const bool one_empty = n_stages_x == n_stages;
+  const int n_stages = pl.stages;
+  const uint32_t stage_bytes = kABytes + pl.boxes * kBoxBytes;
 
   if (threadIdx.x == 0) {
     // full: armed by the leader's producer, completed by both CTAs' TMA bytes (only the leader's copy is used)
     // empty / acc_full: one arrival from the leader's tcgen05.commit, multicast to both CTAs
     // acc_empty: one arrival per epilogue warp of BOTH CTAs, on the leader's copy
-    for (int s = 0; s < kMaxStages; ++s) {
-      mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1);
-      mbar_init(full_x(s), 1); mbar_init(empty_x(s), 1);
-    }
+    for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     mbar_init(acc_full_bar, 1);
     mbar_init(acc_empty_bar, 2 * kEpiWarps);
     mbar_init(fix_bar, 1);
@@ -591,19 +576,19 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
   if (threadIdx.x == 32) CWL_TRACE(1);
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer, right operand (both CTAs)
-    // The whole warp walks the ring; per K block lane 0 arms the barrier, lanes 1..n load one box each, so the copies
-    // of a step go out with one instruction instead of a chain.  The left operand has a ring and a producer of its own
-    // (warp kLeftWarp): it comes out of L2 and needs two or three slots, so the rest of shared memory holds
-    // right-operand bytes in flight, which is what a decode-sized launch is short of.
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    // The whole warp walks the ring; per K block lane 0 arms the barrier and loads the left operand, lanes 1..n
+    // load one right-operand box each, so the copies of a step go out with one instruction instead of a chain.
     {
       uint32_t it_cnt = 0;      // running stage counter across items
       uint32_t s = 0, ph = 0;   // ring slot and phase parity of it_cnt, kept incrementally (no division per step)
       const uint32_t leader_full0 = mapa_shared(full_bar(0), 0);   // full_bar(0) in the leader's shared memory
       bool ok = true;
+      const uint64_t keep_x = policy_evict_last();
       Item item;
       for (int i = 0; ok && get_item(i, pair, sh_begin, p, item); ++i) {
         const bool shrink = item.kind == ITEM_SHRINK;
+        const int m_tile = item.m_pair * 2 + (int)rank;       // this CTA's 128-row tile
         // columns of the right operand this CTA supplies: its half of each MMA's columns (a shrink item runs one
         // MMA of N = R against its projection's A, a projection tile one or two MMAs)
         const int ca = item.wa >> 1, cb = item.wb >> 1;
@@ -611,7 +596,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
         const int col_a = item.n0 + (int)rank * ca;
         const int col_b = item.n0 + item.wa + (int)rank * cb;
         const int n_boxes = boxes_a + boxes_b;
-        const uint32_t tx_pair = 2u * (uint32_t)(n_boxes * kBoxBytes);
+        const uint32_t tx_pair = 2u * (kABytes + n_boxes * kBoxBytes);
         // this lane's box (lanes 1..n_boxes): source matrix in the d_in blocks and in the R blocks, column, slot
         const int bi = lane - 1;
         const bool has_box = bi >= 0 && bi < n_boxes;
@@ -621,15 +606,24 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
         if (has_box) box_x = bi < boxes_a ? col_a + bi * kBoxCols : col_b + (bi - boxes_a) * kBoxCols;
         const int n_blk = item.n_blk0 + item.n_blk1;
         for (int b = 0; b < n_blk; ++b, ++it_cnt) {
-          const bool step_ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag);
+          bool step_ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag);
           const bool phase1 = b >= item.n_blk0;
+          if (phase1 && b == item.n_blk0) {
+            // H' of this CTA's row tile must have been published by whoever finished its shrink
+            if (lane == 0) CWL_TRACE(15);
+            if (lane == 0 && step_ok) step_ok = wait_word(p.flags + m_tile * pl.n_proj + item.proj, p.epoch, 1, abort_flag);
+            if (lane == 0) CWL_TRACE(16);
+            fence_proxy_async();
+          }
           if (!__all_sync(0xffffffffu, step_ok)) { ok = false; break; }
           const int k = phase1 ? (b - item.n_blk0) * BK : (item.kb0 + b) * BK;
-          const uint32_t sb = ring_w + s * stage_bytes;
+          const uint32_t sa = base + s * stage_bytes, sb = sa + kABytes;
           const uint32_t leader_full = leader_full0 + 8u * s;      // this stage's barrier in the leader's shared memory
           if (lane == 0) {
             CWL_TRACE_N(100, it_cnt);
             if (rank == 0) mbar_expect_tx(full_bar(s), tx_pair);
+            if (phase1) tma_load_2d_pair(sa, &tm.h, leader_full, item.proj * p.R + k, m_tile * BM);
+            else tma_load_2d_pair_hint(sa, &tm.x, leader_full, k, m_tile * BM, keep_x);
           } else if (has_box) {
             tma_load_2d_pair(sb + bi * kBoxBytes, phase1 ? map1 : map0, leader_full, box_x, k);
           }
@@ -660,46 +654,6 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
         }
       }
     }
-  } else if (warp == kLeftWarp) {
-    // ------------------------------------------------------------------ TMA producer, left operand (both CTAs)
-    // One thread: this CTA's 128 rows of X for the K blocks of the d_in loop, of H' for those of the R loop.
-    if (lane == 0) {
-      uint32_t it_cnt = 0, s = 0, ph = 0;
-      const uint32_t leader_full0 = mapa_shared(full_x(0), 0);
-      const uint64_t keep_x = policy_evict_last();
-      bool ok = true;
-      Item item;
-      for (int i = 0; ok && get_item(i, pair, sh_begin, p, item); ++i) {
-        const int m_tile = item.m_pair * 2 + (int)rank;       // this CTA's 128-row tile
-        const int n_blk = item.n_blk0 + item.n_blk1;
-        for (int b = 0; b < n_blk; ++b, ++it_cnt) {
-          if (!mbar_wait(one_empty ? empty_bar(s) : empty_x(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-          const bool phase1 = b >= item.n_blk0;
-          if (phase1 && b == item.n_blk0) {
-            // H' of this CTA's row tile must have been published by whoever finished its shrink
-            CWL_TRACE(15);
-            if (!wait_word(p.flags + m_tile * pl.n_proj + item.proj, p.epoch, 1, abort_flag)) { ok = false; break; }
-            CWL_TRACE(16);
-            fence_proxy_async();
-          }
-          const int k = phase1 ? (b - item.n_blk0) * BK : (item.kb0 + b) * BK;
-          const uint32_t sa = base + s * kABytes;
-          const uint32_t leader_full = leader_full0 + 8u * s;
-          if (rank == 0) mbar_expect_tx(full_x(s), 2u * kABytes);
-          if (phase1) tma_load_2d_pair(sa, &tm.h, leader_full, item.proj * p.R + k, m_tile * BM);
-          else tma_load_2d_pair_hint(sa, &tm.x, leader_full, k, m_tile * BM, keep_x);
-          if (++s == (uint32_t)n_stages_x) { s = 0; ph ^= 1u; }
-        }
-      }
-      if (!ok && rank == 0) {
-        // drain: give the copies already issued a bounded chance to land before the CTA leaves
-        for (uint32_t back = 1; back <= (uint32_t)n_stages_x && back <= it_cnt; ++back) {
-          const uint32_t j = it_cnt - back;
-          unsigned long long t0 = global_timer();
-          while (!mbar_try_wait(full_x(j % n_stages_x), (j / n_stages_x) & 1u) && global_timer() - t0 < wait_limit(abort_flag)) {}
-        }
-      }
-    }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
     // One thread issues every MMA of the pair, so the instructions it executes per K block are on the critical path
@@ -710,8 +664,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
     // last block of each phase out once per item.
     if (lane == 0 && rank == 0) {
       uint32_t local = 0;
-      uint32_t s = 0, ph = 0;   // slot and phase parity of the right-operand ring, kept incrementally
-      uint32_t sx = 0, phx = 0; // ... of the left-operand ring
+      uint32_t s = 0, ph = 0;   // ring slot and phase parity, kept incrementally
       bool ok = true;
       Item item;
 #ifdef CWL_TEST_HOOKS
@@ -720,9 +673,8 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
       // descriptors of ring slot 0; a slot is stage_bytes further on (the address field counts 16-byte units and the
       // whole ring lies below 256 KB, so adding to the 64-bit descriptor never carries out of the field)
       const uint64_t desc_a0 = make_smem_desc(base, 16, 1024);
-      const uint64_t desc_b0 = make_smem_desc(ring_w, kBoxBytes, 1024);
+      const uint64_t desc_b0 = make_smem_desc(base + kABytes, kBoxBytes, 1024);
       const uint64_t desc_slot = (uint64_t)(stage_bytes >> 4);
-      constexpr uint64_t desc_slot_x = (uint64_t)(kABytes >> 4);
       constexpr uint64_t kStepA = (UMMA_K * 2) >> 4;        // one K step further in a K-major tile
       constexpr uint64_t kStepB = (UMMA_K * 128) >> 4;      // ... in an N-major box
       uint64_t da = desc_a0, db = desc_b0;
@@ -738,7 +690,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
         const int tail0 = (item.kb0 + item.n_blk0 == pl.nkb0 && (p.d_in & (BK - 1)) != 0) ? (p.d_in & (BK - 1)) / UMMA_K : BK / UMMA_K;
         const int tail1 = (p.R & (BK - 1)) != 0 ? (p.R & (BK - 1)) / UMMA_K : BK / UMMA_K;
         for (int b = 0; b < n_blk; ++b) {
-          if (!mbar_wait(full_x(sx), phx, abort_flag) || !mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
           CWL_TRACE_N(400, blocks_done);
           tc_fence_after();
           int k_steps = BK / UMMA_K;
@@ -763,14 +715,13 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
               if (two) umma_bf16_pair(tmem_base + kMmaN, da + kk * kStepA, db + second + kk * kStepB, idesc_b, kk ? 1u : acc0);
             }
           }
-          if (!one_empty) umma_commit_pair(empty_x(sx));   // frees the slots in both CTAs once these MMAs have read them
-          umma_commit_pair(empty_bar(s));
+          umma_commit_pair(empty_bar(s));            // frees the stage in both CTAs once these MMAs have read it
 #ifdef CWL_TEST_HOOKS
           CWL_TRACE_N(700, blocks_done);
           ++blocks_done;
 #endif
-          if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; db = desc_b0; } else db += desc_slot;
-          if (++sx == (uint32_t)n_stages_x) { sx = 0; phx ^= 1u; da = desc_a0; } else da += desc_slot_x;
+          if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; da = desc_a0; db = desc_b0; }
+          else { da += desc_slot; db += desc_slot; }
         }
         if (ok) umma_commit_pair(acc_full_bar);      // accumulator complete, both CTAs
         CWL_TRACE(2);
@@ -1263,16 +1214,8 @@ Plan search_plan(int T, int d_in, int n_proj, const int* d_out, int R, int pairs
   pl.boxes = tile_boxes(pl.w0);
   if (pl.n_narrow > 0 && tile_boxes(pl.w1) > pl.boxes) pl.boxes = tile_boxes(pl.w1);
   if (R > 0 && boxes_for(R / 2) > pl.boxes) pl.boxes = boxes_for(R / 2);
-  // Ring depths.  The left operand comes out of L2: four slots where that costs the right operand none (prefill:
-  // 4 x 16 KB + 4 x 32 KB), else three; everything else holds right-operand boxes, the bytes HBM has to deliver.
-  {
-    const int ring = pl.split_k > 1 ? kRingBytesSplit : kRingBytes;
-    const int w_slot = pl.boxes * kBoxBytes;
-    const int with4 = (ring - 4 * kABytes) / w_slot, with3 = (ring - 3 * kABytes) / w_slot;
-    pl.stages_x = with3 > with4 && with4 < kMaxStages ? 3 : 4;
-    pl.stages = pl.stages_x == 3 ? with3 : with4;
-    if (pl.stages > kMaxStages) pl.stages = kMaxStages;
-  }
+  pl.stages = (pl.split_k > 1 ? kRingBytesSplit : kRingBytes) / (kABytes + pl.boxes * kBoxBytes);
+  if (pl.stages > kMaxStages) pl.stages = kMaxStages;
 
   // ---- shrink: how finely d_in is split and who does the items.  Items go, one at a time, to the pair with
   // the lightest load so far.  An item costs its K blocks (16 KB of rows + the boxes of A) plus a fixed
