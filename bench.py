@@ -57,7 +57,7 @@ def load_peaks():
 
 # Revision tag of the dominant kernel the ncu counters under profiles/ were taken on.  Bump it whenever
 # cwl_apply's kernel changes: a traffic figure taken on another revision is reported as null.
-APPLY_KERNEL_REVISION = "pairs-256x512-grouped-r10"
+APPLY_KERNEL_REVISION = "pairs-256x512-grouped-r11"
 
 
 def load_traffic(key: str):

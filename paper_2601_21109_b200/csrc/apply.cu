@@ -196,8 +196,9 @@ __device__ __forceinline__ void tma_load_2d_pair_hint(uint32_t dst, const CUtens
       ::"r"(dst), "l"(map), "r"(leader_bar), "r"(x), "r"(y), "l"(policy) : "memory");
 }
 // L2 eviction policies: rows of X are read again by every column tile of their raster group (keep them), rows of Y are
-// written once and not read by this launch (let them go first).  W gets no hint: the pairs that share a column slab read it
-// within a short time of one another, and marking it for early eviction was measured to double its DRAM reads.
+// written once and not read by this launch (let them go first).  W gets no hint when several row tiles share its column slabs:
+// the pairs that share a slab read it within a short time of one another, and marking it for early eviction was measured to
+// double its DRAM reads.  With one row tile (decode) every box is read once and is marked to leave first.
 __device__ __forceinline__ uint64_t policy_evict_last() {
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
@@ -585,6 +586,10 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
       const uint32_t leader_full0 = mapa_shared(full_bar(0), 0);   // full_bar(0) in the leader's shared memory
       bool ok = true;
       const uint64_t keep_x = policy_evict_last();
+      // With a single row tile (decode-sized T) every box of W or A is read by exactly one pair, once: let it leave L2 first,
+      // so that the rows of X, the partial sums and H' stay.  With more row tiles the pairs of a raster group share the box.
+      const bool stream_w = pl.n_m_pairs == 1;
+      const uint64_t drop_w = policy_evict_first();
       Item item;
       for (int i = 0; ok && get_item(i, pair, sh_begin, p, item); ++i) {
         const bool shrink = item.kind == ITEM_SHRINK;
@@ -625,7 +630,8 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
             if (phase1) tma_load_2d_pair(sa, &tm.h, leader_full, item.proj * p.R + k, m_tile * BM);
             else tma_load_2d_pair_hint(sa, &tm.x, leader_full, k, m_tile * BM, keep_x);
           } else if (has_box) {
-            tma_load_2d_pair(sb + bi * kBoxBytes, phase1 ? map1 : map0, leader_full, box_x, k);
+            if (stream_w && !phase1) tma_load_2d_pair_hint(sb + bi * kBoxBytes, map0, leader_full, box_x, k, drop_w);
+            else tma_load_2d_pair(sb + bi * kBoxBytes, phase1 ? map1 : map0, leader_full, box_x, k);
           }
           if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
         }
@@ -1002,6 +1008,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
       if (*epi_last == 0) continue;
       // this CTA completed its projection's share of the row tile: sum the partials, gate, publish H'
       __threadfence();
+      if (threadIdx.x == 64) CWL_TRACE(17);
       const int quads = p.R >> 2;                    // float4 groups per row of this projection
       const int64_t split_stride = (int64_t)2 * pl.n_m_pairs * p.RT * BM;
       // Every thread owns the groups idx = epi_tid + k * 256.  It takes them eight at a time and, split by split, loads
@@ -1028,6 +1035,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
 #pragma unroll
           for (int g = 0; g < kBatch; ++g) { sum[g].x += x[g].x; sum[g].y += x[g].y; sum[g].z += x[g].z; sum[g].w += x[g].w; }
         }
+        if (threadIdx.x == 64) CWL_TRACE(18);
 #pragma unroll
         for (int g = 0; g < kBatch; ++g) {
           if (src[g] == nullptr) continue;

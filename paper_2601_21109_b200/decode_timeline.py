@@ -44,7 +44,8 @@ def describe(t: np.ndarray) -> list:
                      f"+{(t[7] - t[6]) / 1e3:.2f}, their sums copied in +{(t[8] - t[7]) / 1e3:.2f}, reduced and staged +{(t[9] - t[8]) / 1e3:.2f}, "
                      f"Y stored +{(t[3] - t[9]) / 1e3:.2f}")
     if t[11] != 0:
-        tail = f", reduced {us(13):.2f}, fenced {us(14):.2f}" if t[13] > t[12] else " (not the last arriver)"
+        tail = (f", fence passed {us(17):.2f}, partial sums loaded {us(18):.2f}, reduced {us(13):.2f}, fenced {us(14):.2f}"
+                if t[13] > t[12] else " (not the last arriver)")
         lines.append(f"shrink epilogue: accumulator seen {us(5):.2f}, partial sums stored and fenced {us(11):.2f}, arrival counted {us(12):.2f}{tail}")
     return lines
 
