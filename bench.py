@@ -498,7 +498,7 @@ def measure(name: str, args, steps: int, warmup: int, world: int, rank: int, loc
         progress(f"{name}: end to end with host buffers")
         from paper_2601_21109_b200.runner import HostPipeline
         pipe = HostPipeline(w, n_layers=n_layers, grouped=not args.no_group, first=hp, streaming=streaming)
-        e2e_steps = max(4, min(steps, 20))
+        e2e_steps = max(10, min(steps, 20))    # the span includes one un-overlapped upload and download: ten steps keep them under 5 %
         pipe.run(2)
         barrier()
         x, y = pipe.run(e2e_steps)
