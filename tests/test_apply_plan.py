@@ -73,3 +73,29 @@ def test_workspace_grows_with_the_split_and_noalloc_need_does_not():
     for T in (8192, 16384, 32768):                       # the documented reach of the built-in scratch at R = 64
         assert cwl.cwl_apply_noalloc_scratch_need(T, 4096, 11008, 64) <= cwl.NOALLOC_SCRATCH_BYTES
     assert cwl.cwl_apply_noalloc_scratch_need(65536, 4096, 4096, 64) > cwl.NOALLOC_SCRATCH_BYTES
+
+
+def test_a_batch_needs_the_workspaces_of_its_items_on_their_shares_of_the_pairs():
+    # host-only: the decode step's two projections, 37 of the 74 pairs each (equal weight bytes)
+    both = cwl.cwl_apply_batch_workspace_bytes(256, [4096, 11008], [11008, 4096], 64)
+    up = cwl.cwl_apply_batch_workspace_bytes(256, [4096], [11008], 64)
+    down = cwl.cwl_apply_batch_workspace_bytes(256, [11008], [4096], 64)
+    assert both >= 256 and both % 256 == 0 and up % 256 == 0 and down % 256 == 0
+    # alone, an item plans for every pair; in the batch for its share: both are fp32 partial sums + H' + sync words, MBs
+    assert 1 << 20 < both < 1 << 27 and 1 << 18 < up < 1 << 27 and 1 << 18 < down < 1 << 27
+    assert cwl.cwl_apply_batch_workspace_bytes(256, [4096, 11008], [11008, 4096], 64) == both       # deterministic
+    # no adapter: less scratch (no H', no shrink partial sums)
+    assert cwl.cwl_apply_batch_workspace_bytes(256, [4096, 11008], [11008, 4096], 0) <= both
+    # malformed batches answer with the minimum instead of a plan
+    assert cwl.cwl_apply_batch_workspace_bytes(256, [], [], 64) == 256
+    assert cwl.cwl_apply_batch_workspace_bytes(256, [64] * 5, [64] * 5, 64) == 256
+    assert cwl.cwl_apply_batch_workspace_bytes(0, [4096], [4096], 64) == 256
+
+
+def test_a_share_of_the_pairs_changes_the_plan_not_the_coverage():
+    whole = cwl.cwl_apply_plan(256, 4096, 11008, 64, 74)
+    half = cwl.cwl_apply_plan(256, 4096, 11008, 64, 37)
+    assert half["pairs"] <= 37 and whole["pairs"] <= 74
+    assert half["split_k"] == 1 and whole["split_k"] > 1          # 29 whole-K tiles fit 37 pairs; 74 pairs want the K loop split
+    for plan in (whole, half):
+        assert sum(w for _, w in column_tiles(plan, 11008)) == 11008
