@@ -37,6 +37,7 @@ cwl_status cwl_probe_read(const void* ptr, size_t bytes, int32_t* status_word, v
  *   shrink epilogue:   [11] partial sums stored and fenced  [12] arrival counted  [13] reduced (last arriver only)  [14] fenced
  *                      (last arriver, inside the reduce: [17] fence passed  [18] all partial sums loaded and added)
  *   [15],[16] producer: wait for the H' flag begins / ends
+ *   [19],[20],[21] producer: past the wait for the launch ahead, first work item decoded, first ring slot free
  *   K block i of the pair (running count over its items, i < 290): [100+i] loads issued, [400+i] operands landed
  *   (MMA issuer's wait returned), [700+i] MMAs issued and committed.
  * Errors: CUDA. */

@@ -581,6 +581,7 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
     // The whole warp walks the ring; per K block lane 0 arms the barrier and loads the left operand, lanes 1..n
     // load one right-operand box each, so the copies of a step go out with one instruction instead of a chain.
     {
+      if (lane == 0) CWL_TRACE(19);
       uint32_t it_cnt = 0;      // running stage counter across items
       uint32_t s = 0, ph = 0;   // ring slot and phase parity of it_cnt, kept incrementally (no division per step)
       const uint32_t leader_full0 = mapa_shared(full_bar(0), 0);   // full_bar(0) in the leader's shared memory
@@ -610,8 +611,10 @@ __device__ __forceinline__ void apply_body(const GroupMaps& tm, const ApplyParam
         int box_x = 0;
         if (has_box) box_x = bi < boxes_a ? col_a + bi * kBoxCols : col_b + (bi - boxes_a) * kBoxCols;
         const int n_blk = item.n_blk0 + item.n_blk1;
+        if (lane == 0 && it_cnt == 0) CWL_TRACE(20);
         for (int b = 0; b < n_blk; ++b, ++it_cnt) {
           bool step_ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag);
+          if (lane == 0 && it_cnt == 0) CWL_TRACE(21);
           const bool phase1 = b >= item.n_blk0;
           if (phase1 && b == item.n_blk0) {
             // H' of this CTA's row tile must have been published by whoever finished its shrink

@@ -37,6 +37,8 @@ def describe(t: np.ndarray) -> list:
                  f"block period mean {period.mean():.3f} median {np.median(period):.3f}; operands landed -> MMAs committed "
                  f"{(com - full)[4:].mean():.3f}; loads issued -> landed mean {(full - iss)[4:].mean():.2f} min {(full - iss).min():.2f}; "
                  f"last block landed {full[-1]:.2f}; accumulator committed {us(2):.2f}; epilogue done {us(3):.2f}; teardown {us(4):.2f}")
+    if t[19] != 0:
+        lines.append(f"producer: warp past the launch wait {us(19):.2f}, first item decoded {us(20):.2f}, first slot free {us(21):.2f}, first loads issued {iss[0]:.2f}")
     if t[15] != 0:
         lines.append(f"producer waited for H' from {us(15):.2f} to {us(16):.2f}")
     if t[6] != 0:
