@@ -25,6 +25,14 @@ void cwl_debug_set(int64_t wait_limit_ns, int32_t withhold_publish);
  * Errors: INVALID_ARG, CUDA; a wait that runs out flags CWL_ERR_TIMEOUT in *status_word. */
 cwl_status cwl_probe_read(const void* ptr, size_t bytes, int32_t* status_word, void* stream);
 
+/* The same read with the apply kernel's second source mixed in: `ctas` CTAs (1..148) each stream their slice of
+ * [ptr, ptr + bytes) in 16 KB pieces and, with every piece, copy hot_piece bytes from [hot, hot + hot_bytes) at an offset
+ * that is the same in every CTA (as the rows of X are for every column tile), into one ring slot; 192 KB of slots.
+ *   ptr, hot  DEV, 128-byte aligned; hot_piece a multiple of 16, 16..32768; hot_bytes >= hot_piece.
+ * Errors: INVALID_ARG, CUDA; a wait that runs out flags CWL_ERR_TIMEOUT in *status_word. */
+cwl_status cwl_probe_read_mix(const void* ptr, size_t bytes, const void* hot, size_t hot_bytes, uint32_t hot_piece,
+                              int32_t ctas, int32_t* status_word, void* stream);
+
 /* Device timeline of one CTA pair of the apply kernels (any cwl_apply* call made afterwards).  The leader CTA of
  * pair `pair` (blockIdx.x / 2 of the launch; in a batch launch pairs are numbered through all projections) writes
  * %globaltimer readings (ns, 32 ns granularity) into slots[0..1023]; every launch overwrites the slots, so read them

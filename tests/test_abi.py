@@ -36,7 +36,7 @@ def test_library_exports_every_declared_symbol(lib_path):
 def test_the_test_hook_exists_in_the_test_build_only(lib_path):
     from paper_2601_21109_b200 import build
     hooks = ctypes.CDLL(build.LIB_HOOKS)
-    for name in ("cwl_debug_set", "cwl_trace_set", "cwl_probe_read"):
+    for name in ("cwl_debug_set", "cwl_trace_set", "cwl_probe_read", "cwl_probe_read_mix"):
         assert not hasattr(ctypes.CDLL(lib_path), name), name
         assert hasattr(hooks, name), name
     for name in declared_functions():                        # and everything else as well
