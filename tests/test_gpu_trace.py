@@ -45,3 +45,33 @@ def test_a_traced_pair_records_an_ordered_timeline_and_the_result_is_unchanged()
     assert t[0] > 0 and t[0] <= t[1] <= t[400] and t[2] >= t[400 + n - 1] and t[4] >= t[3] >= t[5] >= t[2]
     issued, landed, committed = t[100:100 + n], t[400:400 + n], t[700:700 + n]
     assert (np.diff(landed) >= 0).all() and (issued <= landed).all() and (landed <= committed).all()
+
+
+def test_the_read_probes_of_the_test_build_run_and_refuse_bad_arguments():
+    region = torch.zeros(148 * 16384 * 4, dtype=torch.uint8, device="cuda")
+    hot = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    with cwl.test_hooks() as L:
+        L.cwl_probe_read.restype = C.c_int
+        L.cwl_probe_read.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        L.cwl_probe_read_mix.restype = C.c_int
+        L.cwl_probe_read_mix.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t, C.c_uint32, C.c_int32, C.c_void_p, C.c_void_p]
+        assert L.cwl_probe_read(region.data_ptr(), region.numel(), status.data_ptr(), stream) == 0
+        for ctas, piece in ((148, 10752), (124, 16384), (1, 16)):
+            assert L.cwl_probe_read_mix(region.data_ptr(), region.numel(), hot.data_ptr(), hot.numel(), piece, ctas,
+                                        status.data_ptr(), stream) == 0
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        INVALID = 1
+        assert L.cwl_probe_read(region.data_ptr(), 1000, status.data_ptr(), stream) == INVALID                  # too small
+        assert L.cwl_probe_read_mix(region.data_ptr(), region.numel(), hot.data_ptr(), hot.numel(), 24, 148,
+                                    status.data_ptr(), stream) == INVALID                                       # not a multiple of 16
+        assert L.cwl_probe_read_mix(region.data_ptr(), region.numel(), hot.data_ptr(), hot.numel(), 4096, 149,
+                                    status.data_ptr(), stream) == INVALID                                       # more CTAs than SMs
+        assert L.cwl_probe_read_mix(region.data_ptr(), region.numel(), hot.data_ptr(), 64, 4096, 148,
+                                    status.data_ptr(), stream) == INVALID                                       # hot region smaller than a piece
+        assert L.cwl_probe_read_mix(region.data_ptr() + 16, region.numel() - 16, hot.data_ptr(), hot.numel(), 4096, 148,
+                                    status.data_ptr(), stream) == INVALID                                       # unaligned
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
